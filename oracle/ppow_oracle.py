@@ -1,0 +1,151 @@
+"""ctypes front end of the float64 CPU oracle (``ppow_oracle.c``).
+
+Test infrastructure only: imported by ``tests/``, by the smoke check and by the benchmark's
+CPU-baseline leg.  Nothing in the product package imports this module, and this module imports
+nothing from the product package.
+
+The wrapper only marshals arguments; every number is computed in the C file.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ppow_oracle.c")
+_LIB = os.path.join(_HERE, "libppow_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+F32, BF16 = 0, 1
+GREEDY, STOCHASTIC = 0, 1
+
+POSITION_FIELDS = ("accept_flag", "alpha", "entropy", "kl", "conf", "crit", "logp_tok", "logq_tok",
+                   "logp_max", "target_argmax")
+WINDOW_FIELDS = ("accepted_len", "reward_speedup", "reward_dist", "reward", "delta", "score")
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O2, no fast-math) into a shared object beside its source."""
+    with _lock:
+        stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+        if force or stale:
+            tmp = _LIB + ".tmp.%d" % os.getpid()
+            cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-pthread", "-Wall", "-Wextra",
+                   "-o", tmp, _SRC, "-lm"]
+            subprocess.run(cmd, check=True, capture_output=True, text=True)
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(_LIB)
+        P = ctypes.c_void_p
+        lib.ppow_oracle_score.restype = ctypes.c_int
+        lib.ppow_oracle_score.argtypes = (
+            [ctypes.c_int32] * 5 + [ctypes.c_double] * 4 + [P] * 6 + [P] * 10 + [P] * 6 + [ctypes.c_int32])
+        lib.ppow_oracle_select.restype = ctypes.c_int
+        lib.ppow_oracle_select.argtypes = [P, ctypes.c_int32, ctypes.c_int32, P, P]
+        lib.ppow_oracle_tau_cumprod.restype = ctypes.c_int32
+        lib.ppow_oracle_tau_cumprod.argtypes = [P, ctypes.c_int32]
+        _lib = lib
+    return _lib
+
+
+def _as_numpy_logits(x):
+    """Accept a numpy float32 / uint16(bf16 bits) array or a CPU torch float32 / bfloat16 tensor."""
+    if not isinstance(x, np.ndarray):
+        import torch
+        assert isinstance(x, torch.Tensor) and x.device.type == "cpu"
+        x = x.contiguous()
+        if x.dtype == torch.bfloat16:
+            x = x.view(torch.int16).numpy().view(np.uint16)
+        elif x.dtype == torch.float32:
+            x = x.numpy()
+        else:
+            raise TypeError("logits must be float32 or bfloat16")
+    x = np.ascontiguousarray(x)
+    if x.dtype == np.float32:
+        return x, F32
+    if x.dtype == np.uint16:
+        return x, BF16
+    raise TypeError("logits must be float32 or uint16 (bf16 bit patterns)")
+
+
+def _np(x, dtype):
+    if x is None:
+        return None
+    if not isinstance(x, np.ndarray):
+        x = x.detach().cpu().numpy()
+    return np.ascontiguousarray(x, dtype=dtype)
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def score_windows(draft_logits, target_logits, draft_tokens, *, mode, c, temperature=1.0, eta=1.0,
+                  eps=0.5, uniforms=None, valid_len=None, ref_logp=None, n_threads=None):
+    """Score N windows of K positions over a vocabulary of V entries; returns a dict of numpy arrays.
+
+    Per-position arrays are [N, K]; per-window arrays are [N].  All floating-point results are
+    float64.  ``uniforms`` are float32 values supplied by the caller (App. C.1 draws u_t ~ U(0,1));
+    the oracle draws no random numbers itself.
+    """
+    lib = _load()
+    d, dt_d = _as_numpy_logits(draft_logits)
+    t, dt_t = _as_numpy_logits(target_logits)
+    assert dt_d == dt_t and d.shape == t.shape and d.ndim == 3
+    N, K, V = d.shape
+    tok = _np(draft_tokens, np.int32)
+    assert tok.shape == (N, K)
+    u = _np(uniforms, np.float32)
+    vl = _np(valid_len, np.int32)
+    rl = _np(ref_logp, np.float64)
+    if n_threads is None:
+        n_threads = os.cpu_count() or 1
+    out = {
+        "accept_flag": np.zeros((N, K), np.uint8),
+        "target_argmax": np.zeros((N, K), np.int32),
+        "accepted_len": np.zeros((N,), np.int32),
+    }
+    for f in POSITION_FIELDS:
+        out.setdefault(f, np.zeros((N, K), np.float64))
+    for f in WINDOW_FIELDS:
+        out.setdefault(f, np.zeros((N,), np.float64))
+    rc = lib.ppow_oracle_score(
+        N, K, V, dt_d, int(mode), float(c), float(temperature), float(eta), float(eps),
+        _ptr(d), _ptr(t), _ptr(tok), _ptr(u), _ptr(vl), _ptr(rl),
+        *[_ptr(out[f]) for f in POSITION_FIELDS],
+        *[_ptr(out[f]) for f in WINDOW_FIELDS],
+        int(n_threads))
+    if rc != 0:
+        raise RuntimeError("ppow_oracle_score failed with code %d" % rc)
+    return out
+
+
+def select_windows(score, n_keep, want_mask=False):
+    """Indices of the n_keep largest scores, ordered by (score descending, index ascending)."""
+    lib = _load()
+    s = _np(score, np.float64)
+    N = s.shape[0]
+    sel = np.zeros((max(n_keep, 0),), np.int32)
+    mask = np.zeros((N,), np.uint8) if want_mask else None
+    rc = lib.ppow_oracle_select(_ptr(s), N, int(n_keep), _ptr(sel), _ptr(mask))
+    if rc != 0:
+        raise RuntimeError("ppow_oracle_select failed with code %d" % rc)
+    return (sel, mask) if want_mask else sel
+
+
+def tau_cumprod(flags):
+    """Accepted length by the sum-of-cumulative-products formula of App. C.1."""
+    lib = _load()
+    f = _np(flags, np.uint8)
+    return int(lib.ppow_oracle_tau_cumprod(_ptr(f), int(f.shape[0])))
