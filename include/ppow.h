@@ -1,0 +1,185 @@
+/*
+ * ppow.h -- C ABI of the B200 (sm_100a) PPOW window-scoring library.
+ *
+ * Scores N speculative windows of K drafted positions over a vocabulary of V entries from paired
+ * draft and target logits, then ranks windows for Adaptive Divergence-Aware Windowing.
+ *
+ * Conventions that hold for every entry point unless it says otherwise
+ *   - "device" pointers address memory of the CUDA device that is current when the call is made;
+ *     "host" pointers address ordinary host memory.  The library never takes ownership of a buffer.
+ *   - The library allocates no device memory.  Scratch space is passed in as `workspace`
+ *     (query its size with the matching *_workspace_bytes function; 256-byte alignment required).
+ *   - Calls only enqueue work on `cuda_stream` (a cudaStream_t, NULL = the legacy default stream)
+ *     and return without synchronising.  Inputs are read-only.  Calls on different streams must
+ *     use different workspaces.
+ *   - Host-detectable problems return an error status before anything is launched; nothing is
+ *     printed and the process is never aborted.
+ *   - Logits must be finite.  Layout of logits is [N, K, V] row-major with the vocabulary
+ *     contiguous; per-position arrays are [N, K] row-major; per-window arrays are [N].
+ */
+#ifndef PPOW_H_
+#define PPOW_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PPOW_OK = 0,
+    PPOW_ERR_INVALID_ARG = 1,   /* null/misaligned pointer, size or parameter out of range */
+    PPOW_ERR_UNSUPPORTED = 2,   /* valid request this build cannot serve (e.g. K > 32) */
+    PPOW_ERR_WORKSPACE = 3,     /* workspace missing, misaligned or too small */
+    PPOW_ERR_CUDA = 4,          /* a CUDA runtime call or kernel launch failed */
+    PPOW_ERR_DEVICE_TIMEOUT = 5 /* a bounded device-side wait gave up (reported by ppow_read_error_flags) */
+} ppow_status;
+
+/* Acceptance test.  PPOW_STOCHASTIC is rejection-sampling verification: accept position t iff
+ * u_t <= min(1, P_t(yhat_t)/Q_t(yhat_t)) (App. C.1).  PPOW_GREEDY is its temperature-0 decoding
+ * case: accept iff yhat_t is the target's most likely token (Sec. 5.1 "Temperatures 0.0 / 1.0";
+ * Fig. 1).  The mode changes only the acceptance test; entropy, KL and Delta always use
+ * `temperature`. */
+typedef enum { PPOW_GREEDY = 0, PPOW_STOCHASTIC = 1 } ppow_mode;
+
+typedef enum { PPOW_F32 = 0, PPOW_BF16 = 1 } ppow_dtype;
+
+/* Bits of the device-side error word (ppow_read_error_flags). */
+enum {
+    PPOW_FLAG_TOKEN_RANGE = 1u,   /* some draft token was outside [0, V): that position was rejected */
+    PPOW_FLAG_DEVICE_TIMEOUT = 2u /* a bounded wait inside a kernel ran out */
+};
+
+typedef struct {
+    int32_t N;           /* windows, >= 0 */
+    int32_t K;           /* drafted positions per window, 1..32 (the paper trains with K = 10) */
+    int32_t V;           /* vocabulary size, >= 2 */
+    int32_t dtype;       /* ppow_dtype of both logit tensors */
+    int32_t mode;        /* ppow_mode */
+    float c;             /* relative drafter cost gamma >= 0 in R_speedup = k/(k*gamma + 1) (Sec. 4.3.1) */
+    float temperature;   /* T > 0; P_t = softmax(target/T), Q_t = softmax(draft/T) (Sec. 4.2) */
+    float eta;           /* scale of the Distribution-Based Proximity Reward (Sec. 4.3.2; paper: 1.0) */
+    float eps;           /* its tolerance: R_dist = eta * 1[k = 0] * 1[Delta < eps] (paper: 0.5) */
+} ppow_params;
+
+/* Output buffers, all device memory owned by the caller.  Any pointer except accepted_len may be
+ * NULL, meaning "do not write this output".  Positions t >= valid_len[n] receive 0 in every
+ * per-position output; a window with valid_len[n] == 0 receives 0 in every output. */
+typedef struct {
+    uint8_t *accept_flag;    /* [N,K] result of the per-position acceptance test (not prefix-ANDed) */
+    int32_t *accepted_len;   /* [N]   k = number of leading accepted positions (App. C.1, tau) */
+    float *reward_speedup;   /* [N]   k/(k*c + 1)                                  (Sec. 4.3.1) */
+    float *reward_dist;      /* [N]   eta * 1[k = 0] * 1[Delta < eps]               (Sec. 4.3.2) */
+    float *reward;           /* [N]   reward_speedup + reward_dist                  (Alg. 1, reward line) */
+    float *delta;            /* [N]   proximity gap Delta (see ref_logp below)      (Sec. 4.3.2) */
+    float *score;            /* [N]   s = mean over valid positions of crit         (Sec. 4.2, s_j) */
+    float *kl;               /* [N,K] KL(P_t || Q_t), nats                          (Sec. 4.2) */
+    float *conf;             /* [N,K] C(P_t) = 1 - H(P_t)/ln V, clamped to [0,1]    (Sec. 4.2) */
+    float *crit;             /* [N,K] v_t = C(P_t) * KL(P_t || Q_t)                 (Sec. 4.2; Alg. 1) */
+    float *logp_tok;         /* [N,K] log P_t(yhat_t); -inf for an out-of-range token */
+    float *logq_tok;         /* [N,K] log Q_t(yhat_t); -inf for an out-of-range token */
+    int32_t *target_argmax;  /* [N,K] argmax_v of the stored target logits, lowest index on ties */
+} ppow_outputs;
+
+/* Bytes of device scratch ppow_score_windows needs for these parameters (0 on invalid params). */
+size_t ppow_score_workspace_bytes(const ppow_params *params);
+
+/*
+ * Scoring pass (Sec. 4.2 criticality, App. C.1 verification, Sec. 4.3 rewards; Alg. 1 lines
+ * "Compute criticality score", "Verify", "proximity gap", reward).
+ *
+ *   draft_logits, target_logits  device, [N,K,V] of params->dtype, contiguous.  Both tensors are
+ *                                read from HBM exactly once.
+ *   draft_tokens                 device, [N,K] int32.  A token outside [0,V) is rejected, gets
+ *                                logp_tok = logq_tok = -inf, and sets PPOW_FLAG_TOKEN_RANGE.
+ *   uniforms                     device, [N,K] float32 in [0,1), drawn by the caller;
+ *                                may be NULL iff mode == PPOW_GREEDY.
+ *   valid_len                    device, [N] int32 in [0,K], or NULL for "all K positions valid".
+ *                                Positions t >= valid_len[n] are neither read nor scored.
+ *   ref_logp                     device, [N] float32, or NULL.  If given, it is the target's
+ *                                log-probability of its own reference window and
+ *                                Delta = ref_logp[n] - sum_t log P_t(yhat_t).  If NULL,
+ *                                Delta = sum_t [max_v log P_t(v) - log P_t(yhat_t)], the reference
+ *                                token at each position taken from the same target logits.
+ *   out                          host pointer to a struct of device pointers (read during the call).
+ *   workspace                    device, >= ppow_score_workspace_bytes(params), 256-byte aligned.
+ *                                Contents are undefined afterwards except the error word.
+ *
+ * Returns PPOW_OK once the work is enqueued.  N == 0 is a valid no-op.
+ */
+ppow_status ppow_score_windows(const ppow_params *params,
+                               const void *draft_logits, const void *target_logits,
+                               const int32_t *draft_tokens, const float *uniforms,
+                               const int32_t *valid_len, const float *ref_logp,
+                               const ppow_outputs *out,
+                               void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Same call, with two optional cudaEvent_t handles (NULL = none) that the library records on
+ * `cuda_stream` immediately before and immediately after the row-reduction kernel, the one step of
+ * the pass that streams the logits (Sec. 4.2 softmax/entropy/KL sums).  Lets a caller time that
+ * kernel alone; the events stay owned by the caller. */
+ppow_status ppow_score_windows_traced(const ppow_params *params,
+                                      const void *draft_logits, const void *target_logits,
+                                      const int32_t *draft_tokens, const float *uniforms,
+                                      const int32_t *valid_len, const float *ref_logp,
+                                      const ppow_outputs *out,
+                                      void *workspace, size_t workspace_bytes, void *cuda_stream,
+                                      void *event_reduce_begin, void *event_reduce_end);
+
+/* Copies the error word that the last ppow_score_windows call on `workspace` left behind into
+ * *flags_host (PPOW_FLAG_* bits) and synchronises `cuda_stream` to do so.  Returns
+ * PPOW_ERR_DEVICE_TIMEOUT if that bit is set, PPOW_ERR_CUDA on a CUDA failure, else PPOW_OK. */
+ppow_status ppow_read_error_flags(const void *workspace, uint32_t *flags_host, void *cuda_stream);
+
+/* Bytes of device scratch ppow_select_windows needs for N scores (0 if N <= 0). */
+size_t ppow_select_workspace_bytes(int32_t N);
+
+/*
+ * ADAW window selection (Sec. 4.2: windows with larger s_j are prioritised): writes the indices
+ * of the n_keep largest scores ordered by (score descending, index ascending); equal scores keep
+ * the lower index first, and -0.0 ranks equal to +0.0.  Scores must not be NaN.
+ *
+ *   score      device, [N] float32
+ *   selected   device, [n_keep] int32
+ *   mask       device, [N] uint8 (1 = selected) or NULL
+ *   workspace  device, >= ppow_select_workspace_bytes(N), 256-byte aligned
+ * Requires 0 <= n_keep <= N <= 2^24.  n_keep == 0 or N == 0 is a valid no-op (mask is cleared).
+ */
+ppow_status ppow_select_windows(const float *score, int32_t N, int32_t n_keep,
+                                int32_t *selected, uint8_t *mask,
+                                void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * The whole pass for callers whose buffers are in HOST memory (Alg. 1 lines "Compute criticality
+ * score" through the reward line, followed by the ADAW ranking of Sec. 4.2): stages the windows
+ * through `device_scratch` in chunks of as many windows as fit, scores each chunk, keeps the window
+ * scores on the device, selects the n_keep best of all N windows and copies every requested result
+ * back.  Same arguments as ppow_score_windows + ppow_select_windows except:
+ *   - every input pointer, every pointer inside *out_host, selected_host [n_keep] and mask_host [N]
+ *     (may be NULL) are host pointers; pinned memory lets the copies run asynchronously;
+ *   - device_scratch is device memory, 256-byte aligned, of at least
+ *     ppow_host_scratch_bytes(params, 1) bytes; ppow_host_scratch_bytes(params, N) avoids chunking.
+ * All copies and kernels are enqueued on `cuda_stream`; results are valid once it has been
+ * synchronised.  The token-range error flag is not reported by this entry point (an out-of-range
+ * token still shows as logp_tok = -inf and a rejected position).
+ */
+size_t ppow_host_scratch_bytes(const ppow_params *params, int32_t chunk_windows);
+ppow_status ppow_score_and_select_host(const ppow_params *params,
+                                       const void *draft_logits, const void *target_logits,
+                                       const int32_t *draft_tokens, const float *uniforms,
+                                       const int32_t *valid_len, const float *ref_logp,
+                                       const ppow_outputs *out_host,
+                                       int32_t n_keep, int32_t *selected_host, uint8_t *mask_host,
+                                       void *device_scratch, size_t scratch_bytes, void *cuda_stream);
+
+/* Static, never-NULL description of a status code. */
+const char *ppow_status_string(ppow_status status);
+
+/* Library version as major*10000 + minor*100 + patch. */
+int ppow_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PPOW_H_ */

@@ -1,0 +1,271 @@
+"""ctypes binding of ``libppow.so``: the same entry points as ``include/ppow.h``, marshalling only.
+
+Every step of the scoring path runs in the CUDA library.  There is no CPU or PyTorch fallback: if
+the library has not been built, or a tensor is not on a CUDA device, the call raises.
+PyTorch is used for device memory and streams only.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libppow.so")
+
+PPOW_OK = 0
+PPOW_ERR_INVALID_ARG, PPOW_ERR_UNSUPPORTED, PPOW_ERR_WORKSPACE, PPOW_ERR_CUDA, PPOW_ERR_DEVICE_TIMEOUT = 1, 2, 3, 4, 5
+PPOW_GREEDY, PPOW_STOCHASTIC = 0, 1
+PPOW_F32, PPOW_BF16 = 0, 1
+PPOW_FLAG_TOKEN_RANGE, PPOW_FLAG_DEVICE_TIMEOUT = 1, 2
+
+EXPORTS = ("ppow_score_workspace_bytes", "ppow_score_windows", "ppow_score_windows_traced", "ppow_read_error_flags",
+           "ppow_select_workspace_bytes", "ppow_select_windows", "ppow_host_scratch_bytes",
+           "ppow_score_and_select_host", "ppow_status_string", "ppow_version")
+
+POSITION_OUTPUTS = {"accept_flag": torch.uint8, "kl": torch.float32, "conf": torch.float32, "crit": torch.float32,
+                    "logp_tok": torch.float32, "logq_tok": torch.float32, "target_argmax": torch.int32}
+WINDOW_OUTPUTS = {"accepted_len": torch.int32, "reward_speedup": torch.float32, "reward_dist": torch.float32,
+                  "reward": torch.float32, "delta": torch.float32, "score": torch.float32}
+
+
+class ppow_params(ctypes.Structure):
+    _fields_ = [("N", ctypes.c_int32), ("K", ctypes.c_int32), ("V", ctypes.c_int32),
+                ("dtype", ctypes.c_int32), ("mode", ctypes.c_int32),
+                ("c", ctypes.c_float), ("temperature", ctypes.c_float),
+                ("eta", ctypes.c_float), ("eps", ctypes.c_float)]
+
+
+class ppow_outputs(ctypes.Structure):
+    # field order is the order of the C struct
+    _fields_ = [(n, ctypes.c_void_p) for n in
+                ("accept_flag", "accepted_len", "reward_speedup", "reward_dist", "reward", "delta", "score",
+                 "kl", "conf", "crit", "logp_tok", "logq_tok", "target_argmax")]
+
+
+class PpowError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %s (status %d)" % (where, ppow_status_string(status), status))
+
+
+_lib = None
+
+
+def load_library():
+    """Load libppow.so; raises if it was not built (there is no fallback path)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError("libppow.so is missing: build it with `python -m paper_2605_14978_b200.build` "
+                           "(the scoring path has no CPU or PyTorch fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+    lib.ppow_score_workspace_bytes.restype = sz
+    lib.ppow_score_workspace_bytes.argtypes = [ctypes.POINTER(ppow_params)]
+    lib.ppow_score_windows.restype = ctypes.c_int
+    lib.ppow_score_windows.argtypes = [ctypes.POINTER(ppow_params), vp, vp, vp, vp, vp, vp,
+                                       ctypes.POINTER(ppow_outputs), vp, sz, vp]
+    lib.ppow_score_windows_traced.restype = ctypes.c_int
+    lib.ppow_score_windows_traced.argtypes = lib.ppow_score_windows.argtypes + [vp, vp]
+    lib.ppow_read_error_flags.restype = ctypes.c_int
+    lib.ppow_read_error_flags.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
+    lib.ppow_select_workspace_bytes.restype = sz
+    lib.ppow_select_workspace_bytes.argtypes = [i32]
+    lib.ppow_select_windows.restype = ctypes.c_int
+    lib.ppow_select_windows.argtypes = [vp, i32, i32, vp, vp, vp, sz, vp]
+    lib.ppow_host_scratch_bytes.restype = sz
+    lib.ppow_host_scratch_bytes.argtypes = [ctypes.POINTER(ppow_params), i32]
+    lib.ppow_score_and_select_host.restype = ctypes.c_int
+    lib.ppow_score_and_select_host.argtypes = [ctypes.POINTER(ppow_params), vp, vp, vp, vp, vp, vp,
+                                               ctypes.POINTER(ppow_outputs), i32, vp, vp, vp, sz, vp]
+    lib.ppow_status_string.restype = ctypes.c_char_p
+    lib.ppow_status_string.argtypes = [ctypes.c_int]
+    lib.ppow_version.restype = ctypes.c_int
+    lib.ppow_version.argtypes = []
+    _lib = lib
+    return lib
+
+
+def ppow_status_string(status: int) -> str:
+    return load_library().ppow_status_string(int(status)).decode()
+
+
+def ppow_version() -> int:
+    return int(load_library().ppow_version())
+
+
+def _dev_ptr(t: Optional[torch.Tensor], dtype=None, name="tensor"):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("%s must live on a CUDA device (no CPU path exists)" % name)
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % name)
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError("%s must have dtype %s, got %s" % (name, dtype, t.dtype))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def make_params(N, K, V, dtype, mode, c, temperature=1.0, eta=1.0, eps=0.5) -> ppow_params:
+    return ppow_params(int(N), int(K), int(V), int(dtype), int(mode), float(c), float(temperature),
+                       float(eta), float(eps))
+
+
+def ppow_score_workspace_bytes(params: ppow_params) -> int:
+    return int(load_library().ppow_score_workspace_bytes(ctypes.byref(params)))
+
+
+def ppow_select_workspace_bytes(N: int) -> int:
+    return int(load_library().ppow_select_workspace_bytes(int(N)))
+
+
+def alloc_outputs(N: int, K: int, device) -> dict:
+    out = {k: torch.empty((N, K), dtype=dt, device=device) for k, dt in POSITION_OUTPUTS.items()}
+    out.update({k: torch.empty((N,), dtype=dt, device=device) for k, dt in WINDOW_OUTPUTS.items()})
+    return out
+
+
+def alloc_workspace(nbytes: int, device) -> torch.Tensor:
+    # torch's caching allocator returns 512-byte aligned blocks
+    return torch.empty((max(int(nbytes), 256),), dtype=torch.uint8, device=device)
+
+
+def _event_ptr(ev):
+    """cudaEvent_t of a torch.cuda.Event (created on first record), or NULL."""
+    if ev is None:
+        return None
+    if not ev.cuda_event:
+        ev.record()           # torch creates the CUDA event lazily; the library re-records it
+    return ctypes.c_void_p(ev.cuda_event)
+
+
+def ppow_score_windows(params: ppow_params, draft_logits, target_logits, draft_tokens, uniforms, valid_len,
+                       ref_logp, outputs: dict, workspace: torch.Tensor, stream=None) -> None:
+    """Enqueue the scoring pass; raises PpowError on a non-OK status.  ``outputs`` maps output names
+    to preallocated CUDA tensors (absent or None = not written; ``accepted_len`` is required)."""
+    ppow_score_windows_traced(params, draft_logits, target_logits, draft_tokens, uniforms, valid_len, ref_logp,
+                              outputs, workspace, stream, None, None)
+
+
+def ppow_score_windows_traced(params: ppow_params, draft_logits, target_logits, draft_tokens, uniforms, valid_len,
+                              ref_logp, outputs: dict, workspace: torch.Tensor, stream=None,
+                              event_reduce_begin=None, event_reduce_end=None) -> None:
+    """ppow_score_windows plus two optional torch.cuda.Event objects recorded around the row-reduction kernel."""
+    lib = load_library()
+    lt = torch.float32 if params.dtype == PPOW_F32 else torch.bfloat16
+    o = ppow_outputs()
+    for name, _ in ppow_outputs._fields_:
+        t = outputs.get(name)
+        want = POSITION_OUTPUTS.get(name) or WINDOW_OUTPUTS.get(name)
+        p = _dev_ptr(t, want, name)
+        setattr(o, name, p.value if p is not None else None)
+    traced = event_reduce_begin is not None or event_reduce_end is not None
+    fn = lib.ppow_score_windows_traced if traced else lib.ppow_score_windows
+    extra = (_event_ptr(event_reduce_begin), _event_ptr(event_reduce_end)) if traced else ()
+    st = fn(
+        ctypes.byref(params),
+        _dev_ptr(draft_logits, lt, "draft_logits"), _dev_ptr(target_logits, lt, "target_logits"),
+        _dev_ptr(draft_tokens, torch.int32, "draft_tokens"), _dev_ptr(uniforms, torch.float32, "uniforms"),
+        _dev_ptr(valid_len, torch.int32, "valid_len"), _dev_ptr(ref_logp, torch.float32, "ref_logp"),
+        ctypes.byref(o), _dev_ptr(workspace, torch.uint8, "workspace"),
+        workspace.numel() if workspace is not None else 0, _stream_ptr(stream), *extra)
+    if st != PPOW_OK:
+        raise PpowError(st, "ppow_score_windows")
+
+
+def ppow_read_error_flags(workspace: torch.Tensor, stream=None) -> int:
+    lib = load_library()
+    flags = ctypes.c_uint32(0)
+    st = lib.ppow_read_error_flags(_dev_ptr(workspace, torch.uint8, "workspace"), ctypes.byref(flags),
+                                   _stream_ptr(stream))
+    if st not in (PPOW_OK, PPOW_ERR_DEVICE_TIMEOUT):
+        raise PpowError(st, "ppow_read_error_flags")
+    return int(flags.value)
+
+
+def ppow_select_windows(score, n_keep: int, selected, mask, workspace, stream=None) -> None:
+    lib = load_library()
+    N = int(score.numel()) if score is not None else 0
+    st = lib.ppow_select_windows(
+        _dev_ptr(score, torch.float32, "score"), N, int(n_keep), _dev_ptr(selected, torch.int32, "selected"),
+        _dev_ptr(mask, torch.uint8, "mask"), _dev_ptr(workspace, torch.uint8, "workspace"),
+        workspace.numel() if workspace is not None else 0, _stream_ptr(stream))
+    if st != PPOW_OK:
+        raise PpowError(st, "ppow_select_windows")
+
+
+def _host_ptr(t: Optional[torch.Tensor], dtype=None, name="tensor"):
+    if t is None:
+        return None
+    if t.is_cuda or not t.is_contiguous():
+        raise ValueError("%s must be a contiguous host tensor" % name)
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError("%s must have dtype %s, got %s" % (name, dtype, t.dtype))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def ppow_host_scratch_bytes(params: ppow_params, chunk_windows: int) -> int:
+    return int(load_library().ppow_host_scratch_bytes(ctypes.byref(params), int(chunk_windows)))
+
+
+def ppow_score_and_select_host(params: ppow_params, draft_logits, target_logits, draft_tokens, uniforms, valid_len,
+                               ref_logp, outputs_host: dict, n_keep: int, selected_host, mask_host,
+                               device_scratch: torch.Tensor, stream=None) -> None:
+    """Host-buffer entry point: all tensors except ``device_scratch`` are host tensors (pinned for async copies)."""
+    lib = load_library()
+    lt = torch.float32 if params.dtype == PPOW_F32 else torch.bfloat16
+    o = ppow_outputs()
+    for name, _ in ppow_outputs._fields_:
+        want = POSITION_OUTPUTS.get(name) or WINDOW_OUTPUTS.get(name)
+        p = _host_ptr(outputs_host.get(name), want, name)
+        setattr(o, name, p.value if p is not None else None)
+    st = lib.ppow_score_and_select_host(
+        ctypes.byref(params), _host_ptr(draft_logits, lt, "draft_logits"), _host_ptr(target_logits, lt, "target_logits"),
+        _host_ptr(draft_tokens, torch.int32, "draft_tokens"), _host_ptr(uniforms, torch.float32, "uniforms"),
+        _host_ptr(valid_len, torch.int32, "valid_len"), _host_ptr(ref_logp, torch.float32, "ref_logp"),
+        ctypes.byref(o), int(n_keep), _host_ptr(selected_host, torch.int32, "selected_host"),
+        _host_ptr(mask_host, torch.uint8, "mask_host"), _dev_ptr(device_scratch, torch.uint8, "device_scratch"),
+        device_scratch.numel(), _stream_ptr(stream))
+    if st != PPOW_OK:
+        raise PpowError(st, "ppow_score_and_select_host")
+
+
+# ---- convenience wrappers (allocation + the calls above; no arithmetic) -----------------------
+
+
+def score_windows(draft_logits, target_logits, draft_tokens, *, mode, c, temperature=1.0, eta=1.0, eps=0.5,
+                  uniforms=None, valid_len=None, ref_logp=None, stream=None) -> dict:
+    """Allocate outputs and workspace, run ppow_score_windows, return the dict of output tensors."""
+    N, K, V = draft_logits.shape
+    dt = PPOW_F32 if draft_logits.dtype == torch.float32 else PPOW_BF16
+    params = make_params(N, K, V, dt, mode, c, temperature, eta, eps)
+    dev = draft_logits.device
+    with torch.cuda.device(dev):
+        out = alloc_outputs(N, K, dev)
+        ws = alloc_workspace(ppow_score_workspace_bytes(params), dev)
+        ppow_score_windows(params, draft_logits, target_logits, draft_tokens, uniforms, valid_len, ref_logp, out,
+                           ws, stream)
+    out["_workspace"] = ws
+    return out
+
+
+def select_windows(score, n_keep: int, want_mask: bool = False, stream=None):
+    """Allocate and run ppow_select_windows; returns selected indices (and the mask if asked)."""
+    N = int(score.numel())
+    dev = score.device
+    with torch.cuda.device(dev):
+        sel = torch.empty((max(int(n_keep), 0),), dtype=torch.int32, device=dev)
+        mask = torch.empty((N,), dtype=torch.uint8, device=dev) if want_mask else None
+        ws = alloc_workspace(ppow_select_workspace_bytes(N), dev)
+        ppow_select_windows(score, n_keep, sel, mask, ws, stream)
+    return (sel, mask) if want_mask else sel

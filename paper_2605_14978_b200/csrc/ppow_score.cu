@@ -1,0 +1,505 @@
+// PPOW scoring pass: row-reduction kernels (the only HBM-heavy step), the per-window scan kernel,
+// and the host entry points ppow_score_windows / ppow_score_workspace_bytes / ppow_read_error_flags.
+#include "../../include/ppow.h"
+#include "ppow_device.cuh"
+
+#include <math.h>
+
+namespace ppow {
+
+constexpr int ROW_THREADS = 256;   // threads per CTA in the row-reduction kernels
+constexpr int ROW_WARPS = ROW_THREADS / 32;
+constexpr int UNROLL = 4;          // 16-byte units per thread per tensor in flight
+constexpr int MAX_SEGMENTS = 16;   // a row is split into at most this many work items
+constexpr size_t WS_HEADER_BYTES = 256;
+
+// Workspace header (first WS_HEADER_BYTES of the workspace).
+struct WsHeader {
+    unsigned int next_item;    // dynamic work counter of the row-reduction kernel
+    unsigned int error_flags;  // PPOW_FLAG_* bits
+};
+
+struct RowJob {
+    const void *target, *draft;
+    const int32_t *valid_len;
+    RowPartial *partials;      // [N*K*segments]
+    WsHeader *header;
+    int32_t N, K, V;
+    int32_t segments;          // work items per row
+    uint32_t total_items;      // N*K*segments
+    float s;                   // log2(e)/T
+};
+
+// ---- work distribution -----------------------------------------------------------------------
+// Items are handed out by an atomic counter so that ragged windows (rows beyond valid_len are
+// never read) and the tail of the launch stay balanced.  Thread 0 fetches the next valid item
+// while the CTA is busy with the current one.
+
+__device__ __forceinline__ bool item_is_valid(const RowJob &job, uint32_t item)
+{
+    if (job.valid_len == nullptr) return true;
+    const uint32_t row = item / (uint32_t)job.segments;
+    const int32_t n = (int32_t)(row / (uint32_t)job.K), k = (int32_t)(row % (uint32_t)job.K);
+    return k < __ldg(job.valid_len + n);
+}
+
+__device__ __forceinline__ uint32_t fetch_item(const RowJob &job)
+{
+    uint32_t it;
+    do {
+        it = atomicAdd(&job.header->next_item, 1u);
+    } while (it < job.total_items && !item_is_valid(job, it));
+    return it;
+}
+
+// Block-level merge of per-warp partials; result written by thread 0.
+__device__ __forceinline__ void block_merge_and_store(const RowPartial &wp, RowPartial *smem_parts,
+                                                      RowPartial *dst)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) smem_parts[warp] = wp;
+    __syncthreads();
+    if (warp == 0) {
+        RowAcc acc;
+        int32_t arg = INT32_MAX;
+        if (lane < ROW_WARPS) {
+            acc = acc_from_partial(smem_parts[lane]);
+            arg = smem_parts[lane].argmax;
+        } else {
+            acc.reset();
+        }
+        RowPartial p = warp_reduce(acc, arg);
+        if (lane == 0) *dst = p;
+    }
+}
+
+// ---- bf16, 16-byte vector path -----------------------------------------------------------------
+// Requires V % 8 == 0 and 16-byte aligned tensors.  Each thread streams 16-byte units
+// u = u0 + tid + j*ROW_THREADS with UNROLL loads per tensor in flight; both tensors are read once.
+
+template <int NU>
+__device__ __forceinline__ void bf16_group(const uint4 *__restrict__ pa, const uint4 *__restrict__ pb,
+                                           int32_t u, RowAcc &acc, float s)
+{
+    uint4 A[NU], B[NU];
+#pragma unroll
+    for (int j = 0; j < NU; ++j) A[j] = __ldcs(pa + u + j * ROW_THREADS);
+#pragma unroll
+    for (int j = 0; j < NU; ++j) B[j] = __ldcs(pb + u + j * ROW_THREADS);
+
+    uint32_t ma = max_bf16x2(max_bf16x2(A[0].x, A[0].y), max_bf16x2(A[0].z, A[0].w));
+    uint32_t mb = max_bf16x2(max_bf16x2(B[0].x, B[0].y), max_bf16x2(B[0].z, B[0].w));
+#pragma unroll
+    for (int j = 1; j < NU; ++j) {
+        ma = max_bf16x2(ma, max_bf16x2(max_bf16x2(A[j].x, A[j].y), max_bf16x2(A[j].z, A[j].w)));
+        mb = max_bf16x2(mb, max_bf16x2(max_bf16x2(B[j].x, B[j].y), max_bf16x2(B[j].z, B[j].w)));
+    }
+    const float tmax_a = fmaxf(bf16_lo(ma), bf16_hi(ma));
+    const float tmax_b = fmaxf(bf16_lo(mb), bf16_hi(mb));
+    acc.guard(tmax_a, tmax_b, s);
+    if (tmax_a > acc.max_a) {   // strict: an equal value seen later has a higher index
+        acc.max_a = tmax_a;
+        acc.best = u * 8 + NU;  // unit index and group size packed: (u << 3) | NU, NU in {1, 4}
+    }
+#pragma unroll
+    for (int j = 0; j < NU; ++j) {
+        acc.add_word(A[j].x, B[j].x, s);
+        acc.add_word(A[j].y, B[j].y, s);
+        acc.add_word(A[j].z, B[j].z, s);
+        acc.add_word(A[j].w, B[j].w, s);
+    }
+    acc.flush();
+}
+
+__global__ void __launch_bounds__(ROW_THREADS, 4) row_reduce_bf16_vec_kernel(const RowJob job)
+{
+    __shared__ RowPartial s_parts[ROW_WARPS];
+    __shared__ uint32_t s_item[2];
+
+    const int tid = threadIdx.x;
+    const int32_t units_per_row = job.V >> 3;
+    if (tid == 0) s_item[0] = fetch_item(job);
+    __syncthreads();
+    uint32_t item = s_item[0];
+    int buf = 0;
+
+    while (item < job.total_items) {
+        if (tid == 0) s_item[buf ^ 1] = fetch_item(job);   // prefetch the next item
+
+        const uint32_t row = item / (uint32_t)job.segments;
+        const int32_t seg = (int32_t)(item % (uint32_t)job.segments);
+        const int32_t u0 = (int32_t)(((int64_t)units_per_row * seg) / job.segments);
+        const int32_t u1 = (int32_t)(((int64_t)units_per_row * (seg + 1)) / job.segments);
+        const uint4 *pa = reinterpret_cast<const uint4 *>(job.target) + (size_t)row * units_per_row;
+        const uint4 *pb = reinterpret_cast<const uint4 *>(job.draft) + (size_t)row * units_per_row;
+
+        RowAcc acc;
+        acc.reset();
+        int32_t u = u0 + tid;
+        for (; u + (UNROLL - 1) * ROW_THREADS < u1; u += UNROLL * ROW_THREADS)
+            bf16_group<UNROLL>(pa, pb, u, acc, job.s);
+        for (; u < u1; u += ROW_THREADS)
+            bf16_group<1>(pa, pb, u, acc, job.s);
+
+        // lowest vocabulary index of this thread's maximum: rescan the group that raised it
+        int32_t arg = INT32_MAX;
+        if (acc.max_a > -INFINITY) {
+            const int32_t bu = acc.best >> 3, bn = acc.best & 7;
+            for (int j = 0; j < bn && arg == INT32_MAX; ++j) {
+                const uint4 w4 = __ldg(pa + bu + j * ROW_THREADS);
+                const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+                for (int q = 3; q >= 0; --q) {
+                    if (bf16_hi(w[q]) == acc.max_a) arg = (bu + j * ROW_THREADS) * 8 + 2 * q + 1;
+                    if (bf16_lo(w[q]) == acc.max_a) arg = (bu + j * ROW_THREADS) * 8 + 2 * q;
+                }
+            }
+        }
+        const RowPartial wp = warp_reduce(acc, arg);
+        block_merge_and_store(wp, s_parts, job.partials + item);
+        __syncthreads();   // s_parts and s_item[buf^1] are stable past this point
+        buf ^= 1;
+        item = s_item[buf];
+    }
+}
+
+// ---- generic path: any V, any alignment, f32 or bf16 -------------------------------------------
+
+template <typename T>
+__device__ __forceinline__ float load_logit(const T *p, size_t i);
+template <>
+__device__ __forceinline__ float load_logit<float>(const float *p, size_t i) { return __ldcs(p + i); }
+template <>
+__device__ __forceinline__ float load_logit<uint16_t>(const uint16_t *p, size_t i)
+{
+    return __uint_as_float(((uint32_t)__ldcs(p + i)) << 16);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(ROW_THREADS, 4) row_reduce_generic_kernel(const RowJob job)
+{
+    __shared__ RowPartial s_parts[ROW_WARPS];
+    __shared__ uint32_t s_item[2];
+
+    const int tid = threadIdx.x;
+    if (tid == 0) s_item[0] = fetch_item(job);
+    __syncthreads();
+    uint32_t item = s_item[0];
+    int buf = 0;
+
+    while (item < job.total_items) {
+        if (tid == 0) s_item[buf ^ 1] = fetch_item(job);
+
+        const uint32_t row = item / (uint32_t)job.segments;
+        const int32_t seg = (int32_t)(item % (uint32_t)job.segments);
+        const int32_t v0 = (int32_t)(((int64_t)job.V * seg) / job.segments);
+        const int32_t v1 = (int32_t)(((int64_t)job.V * (seg + 1)) / job.segments);
+        const T *pa = reinterpret_cast<const T *>(job.target) + (size_t)row * job.V;
+        const T *pb = reinterpret_cast<const T *>(job.draft) + (size_t)row * job.V;
+
+        RowAcc acc;
+        acc.reset();
+        int32_t arg = INT32_MAX;
+        for (int32_t v = v0 + tid; v < v1; v += ROW_THREADS) {
+            const float a = load_logit<T>(pa, v), b = load_logit<T>(pb, v);
+            acc.guard(a, b, job.s);
+            if (a > acc.max_a) { acc.max_a = a; arg = v; }
+            acc.add_pair(a, b, job.s, 0);
+            acc.flush();
+        }
+        const RowPartial wp = warp_reduce(acc, arg);
+        block_merge_and_store(wp, s_parts, job.partials + item);
+        __syncthreads();
+        buf ^= 1;
+        item = s_item[buf];
+    }
+}
+
+// ---- per-window scan: float64 epilogue per position, prefix scan, rewards, score --------------
+
+struct ScanJob {
+    const void *target, *draft;
+    const int32_t *tokens;
+    const float *uniforms;
+    const int32_t *valid_len;
+    const float *ref_logp;
+    const RowPartial *partials;
+    WsHeader *header;
+    ppow_outputs out;
+    int32_t N, K, V, dtype, mode, segments;
+    float s;         // log2(e)/T as used by the row reduction
+    float c, eta, eps;
+};
+
+__device__ __forceinline__ double raw_logit(const void *base, int32_t dtype, size_t idx)
+{
+    if (dtype == PPOW_F32) return (double)__ldg(reinterpret_cast<const float *>(base) + idx);
+    return (double)__uint_as_float(((uint32_t)__ldg(reinterpret_cast<const uint16_t *>(base) + idx)) << 16);
+}
+
+__device__ __forceinline__ double warp_sum_f64(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+constexpr int SCAN_THREADS = 128;
+
+__global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob job)
+{
+    const int lane = threadIdx.x & 31;
+    const int32_t n = (int32_t)((blockIdx.x * (unsigned)SCAN_THREADS + threadIdx.x) >> 5);
+    if (n >= job.N) return;
+    const int32_t K = job.K;
+    int32_t L = job.valid_len ? __ldg(job.valid_len + n) : K;
+    L = max(0, min(L, K));
+    const bool active = lane < L;
+    const double LN2 = 0.69314718055994530942;
+
+    double crit = 0.0, gap = 0.0, lp = 0.0;
+    float o_kl = 0.f, o_conf = 0.f, o_crit = 0.f, o_lp = 0.f, o_lq = 0.f;
+    int32_t o_arg = 0;
+    int flag = 0;
+
+    if (active) {
+        const size_t row = (size_t)n * K + lane;
+        // merge this row's partials against the largest references
+        const RowPartial *pp = job.partials + row * job.segments;
+        double Ra = -INFINITY, Rb = -INFINITY;
+        float mx = -INFINITY;
+        for (int i = 0; i < job.segments; ++i) {
+            Ra = fmax(Ra, (double)pp[i].rho_a);
+            Rb = fmax(Rb, (double)pp[i].rho_b);
+            mx = fmaxf(mx, pp[i].max_a);
+        }
+        double Sa = 0.0, Sb = 0.0, E = 0.0, D = 0.0;
+        int32_t arg = INT32_MAX;
+        for (int i = 0; i < job.segments; ++i) {
+            const RowPartial p = pp[i];
+            const double da = (double)p.rho_a - Ra, db = (double)p.rho_b - Rb;
+            const double fa = exp2(da), fb = exp2(db);
+            const double pSa = (double)p.Sa + (double)p.Sa_lo, pSb = (double)p.Sb + (double)p.Sb_lo;
+            const double sa = fa * pSa;
+            Sa += sa;
+            E += fa * ((double)p.E + da * pSa);
+            D += fa * ((double)p.D + (da - db) * pSa);
+            Sb += fb * pSb;
+            if (p.max_a == mx) arg = min(arg, p.argmax);
+        }
+        const double s = (double)job.s;
+        const double l2Sa = log2(Sa), l2Sb = log2(Sb);
+        const double H = (l2Sa - E / Sa) * LN2;                 // entropy of P, nats
+        const double KL = (D / Sa - l2Sa + l2Sb) * LN2;         // KL(P || Q), nats
+        double C = 1.0 - H / log((double)job.V);
+        C = fmin(1.0, fmax(0.0, C));
+        crit = C * KL;
+        const double lmax = (((double)mx * s - Ra) - l2Sa) * LN2;
+
+        const int32_t tok = __ldg(job.tokens + row);
+        double lq;
+        if (tok < 0 || tok >= job.V) {
+            atomicOr(&job.header->error_flags, (unsigned)PPOW_FLAG_TOKEN_RANGE);
+            lp = -INFINITY;
+            lq = -INFINITY;
+            flag = 0;
+        } else {
+            const double a_tok = raw_logit(job.target, job.dtype, row * job.V + tok);
+            const double b_tok = raw_logit(job.draft, job.dtype, row * job.V + tok);
+            lp = ((a_tok * s - Ra) - l2Sa) * LN2;
+            lq = ((b_tok * s - Rb) - l2Sb) * LN2;
+            if (job.mode == PPOW_GREEDY) {
+                flag = (tok == arg);
+            } else {
+                const double alpha = fmin(1.0, exp(lp - lq));
+                flag = ((double)__ldg(job.uniforms + row) <= alpha);
+            }
+        }
+        gap = lmax - lp;
+        o_kl = (float)KL; o_conf = (float)C; o_crit = (float)crit; o_lp = (float)lp; o_lq = (float)lq;
+        o_arg = arg;
+    }
+
+    if (lane < K) {
+        const size_t row = (size_t)n * K + lane;
+        if (job.out.accept_flag) job.out.accept_flag[row] = (uint8_t)flag;
+        if (job.out.kl) job.out.kl[row] = o_kl;
+        if (job.out.conf) job.out.conf[row] = o_conf;
+        if (job.out.crit) job.out.crit[row] = o_crit;
+        if (job.out.logp_tok) job.out.logp_tok[row] = o_lp;
+        if (job.out.logq_tok) job.out.logq_tok[row] = o_lq;
+        if (job.out.target_argmax) job.out.target_argmax[row] = o_arg;
+    }
+
+    // accepted length = number of leading accepted positions (App. C.1)
+    const unsigned accepted = __ballot_sync(0xffffffffu, flag != 0);
+    const unsigned valid_mask = (L >= 32) ? 0xffffffffu : ((1u << L) - 1u);
+    const unsigned rejected = (~accepted) & valid_mask;
+    const int32_t k = rejected ? (__ffs(rejected) - 1) : L;
+
+    const double sum_crit = warp_sum_f64(crit);
+    const double sum_gap = warp_sum_f64(gap);
+    const double sum_lp = warp_sum_f64(lp);
+
+    if (lane == 0) {
+        float r_speed = 0.f, r_dist = 0.f, delta = 0.f, score = 0.f;
+        if (L > 0) {
+            const double rs = (double)k / ((double)k * (double)job.c + 1.0);
+            const double dl = job.ref_logp ? ((double)__ldg(job.ref_logp + n) - sum_lp) : sum_gap;
+            r_speed = (float)rs;
+            delta = (float)dl;
+            r_dist = (k == 0 && dl < (double)job.eps) ? job.eta : 0.f;
+            score = (float)(sum_crit / (double)L);
+        }
+        job.out.accepted_len[n] = k;
+        if (job.out.reward_speedup) job.out.reward_speedup[n] = r_speed;
+        if (job.out.reward_dist) job.out.reward_dist[n] = r_dist;
+        if (job.out.reward) job.out.reward[n] = r_speed + r_dist;
+        if (job.out.delta) job.out.delta[n] = delta;
+        if (job.out.score) job.out.score[n] = score;
+    }
+}
+
+// ---- host side ----------------------------------------------------------------------------------
+
+static bool params_ok(const ppow_params *p)
+{
+    if (!p) return false;
+    if (p->N < 0 || p->K < 1 || p->V < 2) return false;
+    if (p->dtype != PPOW_F32 && p->dtype != PPOW_BF16) return false;
+    if (p->mode != PPOW_GREEDY && p->mode != PPOW_STOCHASTIC) return false;
+    if (!(p->temperature > 0.0f) || !isfinite(p->temperature)) return false;
+    if (!(p->c >= 0.0f) || !isfinite(p->c)) return false;
+    if (!isfinite(p->eta) || !isfinite(p->eps)) return false;
+    if ((int64_t)p->N * p->K > (int64_t)1 << 26) return false;   // rows * MAX_SEGMENTS must fit 32 bits
+    return true;
+}
+
+// Work items per row: one for large launches, more when there are too few rows to fill the GPU.
+// Depends only on (N, K, V) so that the workspace size is a pure function of the parameters.
+static int segments_for(const ppow_params *p)
+{
+    const int64_t rows = (int64_t)p->N * p->K;
+    if (rows <= 0) return 1;
+    const int64_t want_items = 148 * 4 * 8;   // ~8 items per resident CTA on a B200
+    int64_t seg = (want_items + rows - 1) / rows;
+    const int64_t elems_min = 4096;            // do not cut a row finer than this many logits
+    const int64_t seg_cap = p->V / elems_min > 1 ? p->V / elems_min : 1;
+    if (seg > seg_cap) seg = seg_cap;
+    if (seg > MAX_SEGMENTS) seg = MAX_SEGMENTS;
+    if (seg < 1) seg = 1;
+    return (int)seg;
+}
+
+}  // namespace ppow
+
+using namespace ppow;
+
+extern "C" size_t ppow_score_workspace_bytes(const ppow_params *params)
+{
+    if (!params_ok(params) || params->K > 32) return 0;
+    const size_t rows = (size_t)params->N * params->K;
+    return WS_HEADER_BYTES + rows * segments_for(params) * sizeof(RowPartial);
+}
+
+extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
+                                                 const void *draft_logits, const void *target_logits,
+                                                 const int32_t *draft_tokens, const float *uniforms,
+                                                 const int32_t *valid_len, const float *ref_logp,
+                                                 const ppow_outputs *out,
+                                                 void *workspace, size_t workspace_bytes, void *cuda_stream,
+                                                 void *event_reduce_begin, void *event_reduce_end)
+{
+    if (!params_ok(params) || !out) return PPOW_ERR_INVALID_ARG;
+    if (params->K > 32) return PPOW_ERR_UNSUPPORTED;
+    if (params->N == 0) return PPOW_OK;
+    if (!draft_logits || !target_logits || !draft_tokens || !out->accepted_len) return PPOW_ERR_INVALID_ARG;
+    if (params->mode == PPOW_STOCHASTIC && !uniforms) return PPOW_ERR_INVALID_ARG;
+    const size_t esize = params->dtype == PPOW_F32 ? 4 : 2;
+    if (((uintptr_t)draft_logits % esize) || ((uintptr_t)target_logits % esize)) return PPOW_ERR_INVALID_ARG;
+    const size_t need = ppow_score_workspace_bytes(params);
+    if (!workspace || ((uintptr_t)workspace % 256) || workspace_bytes < need) return PPOW_ERR_WORKSPACE;
+
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    WsHeader *header = (WsHeader *)workspace;
+    RowPartial *partials = (RowPartial *)((char *)workspace + WS_HEADER_BYTES);
+    if (cudaMemsetAsync(header, 0, WS_HEADER_BYTES, stream) != cudaSuccess) return PPOW_ERR_CUDA;
+
+    const int segments = segments_for(params);
+    const float s = (float)(1.4426950408889634074 / (double)params->temperature);
+
+    RowJob rj;
+    rj.target = target_logits; rj.draft = draft_logits; rj.valid_len = valid_len;
+    rj.partials = partials; rj.header = header;
+    rj.N = params->N; rj.K = params->K; rj.V = params->V;
+    rj.segments = segments;
+    rj.total_items = (uint32_t)((size_t)params->N * params->K * segments);
+    rj.s = s;
+
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return PPOW_ERR_CUDA;
+
+    const bool vec_ok = params->dtype == PPOW_BF16 && (params->V % 8 == 0) &&
+                        ((uintptr_t)draft_logits % 16 == 0) && ((uintptr_t)target_logits % 16 == 0) &&
+                        (params->V / 8 >= segments);
+    int per_sm = 0;
+    cudaError_t e;
+    if (vec_ok)
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_reduce_bf16_vec_kernel, ROW_THREADS, 0);
+    else if (params->dtype == PPOW_BF16)
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_reduce_generic_kernel<uint16_t>, ROW_THREADS, 0);
+    else
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_reduce_generic_kernel<float>, ROW_THREADS, 0);
+    if (e != cudaSuccess || per_sm < 1) return PPOW_ERR_CUDA;
+    unsigned grid = (unsigned)(sms * per_sm);
+    if (grid > rj.total_items) grid = rj.total_items;
+
+    if (event_reduce_begin && cudaEventRecord((cudaEvent_t)event_reduce_begin, stream) != cudaSuccess)
+        return PPOW_ERR_CUDA;
+    if (vec_ok)
+        row_reduce_bf16_vec_kernel<<<grid, ROW_THREADS, 0, stream>>>(rj);
+    else if (params->dtype == PPOW_BF16)
+        row_reduce_generic_kernel<uint16_t><<<grid, ROW_THREADS, 0, stream>>>(rj);
+    else
+        row_reduce_generic_kernel<float><<<grid, ROW_THREADS, 0, stream>>>(rj);
+    if (cudaGetLastError() != cudaSuccess) return PPOW_ERR_CUDA;
+    if (event_reduce_end && cudaEventRecord((cudaEvent_t)event_reduce_end, stream) != cudaSuccess)
+        return PPOW_ERR_CUDA;
+
+    ScanJob sj;
+    sj.target = target_logits; sj.draft = draft_logits; sj.tokens = draft_tokens; sj.uniforms = uniforms;
+    sj.valid_len = valid_len; sj.ref_logp = ref_logp; sj.partials = partials; sj.header = header;
+    sj.out = *out;
+    sj.N = params->N; sj.K = params->K; sj.V = params->V; sj.dtype = params->dtype; sj.mode = params->mode;
+    sj.segments = segments; sj.s = s; sj.c = params->c; sj.eta = params->eta; sj.eps = params->eps;
+    const unsigned scan_grid = (unsigned)(((size_t)params->N * 32 + SCAN_THREADS - 1) / SCAN_THREADS);
+    window_scan_kernel<<<scan_grid, SCAN_THREADS, 0, stream>>>(sj);
+    if (cudaGetLastError() != cudaSuccess) return PPOW_ERR_CUDA;
+    return PPOW_OK;
+}
+
+extern "C" ppow_status ppow_score_windows(const ppow_params *params,
+                                          const void *draft_logits, const void *target_logits,
+                                          const int32_t *draft_tokens, const float *uniforms,
+                                          const int32_t *valid_len, const float *ref_logp,
+                                          const ppow_outputs *out,
+                                          void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    return ppow_score_windows_traced(params, draft_logits, target_logits, draft_tokens, uniforms, valid_len,
+                                     ref_logp, out, workspace, workspace_bytes, cuda_stream, nullptr, nullptr);
+}
+
+extern "C" ppow_status ppow_read_error_flags(const void *workspace, uint32_t *flags_host, void *cuda_stream)
+{
+    if (!workspace || !flags_host) return PPOW_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const WsHeader *header = (const WsHeader *)workspace;
+    unsigned int v = 0;
+    if (cudaMemcpyAsync(&v, &header->error_flags, sizeof v, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return PPOW_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return PPOW_ERR_CUDA;
+    *flags_host = v;
+    return (v & PPOW_FLAG_DEVICE_TIMEOUT) ? PPOW_ERR_DEVICE_TIMEOUT : PPOW_OK;
+}

@@ -1,0 +1,292 @@
+"""GPU-vs-oracle parity through the C ABI on the five synthetic workloads and on edge cases."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_14978_b200 import binding as B
+from paper_2605_14978_b200 import workloads as W
+
+from parity_util import compare_scores, compare_selection, run_gpu, run_oracle
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+# (workload index, windows used for the element-by-element comparison)
+SMALL = [(0, 64), (1, 96), (2, 48), (3, 80), (4, 24)]
+
+
+def _check_workload(w, x, sample=None):
+    reports = {}
+    for mode in w.modes:
+        gpu = run_gpu(x, mode, w.c, w.temperature)
+        assert B.ppow_read_error_flags(gpu["_workspace"]) == 0
+        ref = run_oracle(x, mode, w.c, w.temperature, windows=sample)
+        rep = compare_scores(gpu, ref, mode, x["uniforms"], windows=sample)
+        if sample is None:
+            rep.update(compare_selection(gpu["score"], w.n_keep, ref["score"]))
+        else:
+            rep.update(compare_selection(gpu["score"], w.n_keep))
+        # properties that hold at any size
+        L = x["valid_len"] if x["valid_len"] is not None else torch.full((w.N,), w.K, device=DEV, dtype=torch.int32)
+        assert bool(((gpu["accepted_len"] >= 0) & (gpu["accepted_len"] <= L)).all())
+        assert bool((gpu["conf"] >= 0).all()) and bool((gpu["conf"] <= 1).all())
+        assert bool((gpu["kl"] >= -1e-5).all())
+        assert bool(torch.isfinite(gpu["score"]).all())
+        # run-to-run determinism (catches races in the reductions)
+        again = run_gpu(x, mode, w.c, w.temperature)
+        for k, v in gpu.items():
+            if not k.startswith("_"):
+                assert torch.equal(v, again[k]), k
+        reports[mode] = rep
+    return reports
+
+
+@pytest.mark.parametrize("idx,n", SMALL)
+def test_workload_reduced_windows_elementwise(idx, n):
+    w = W.scaled(W.WORKLOADS[idx], n)
+    x = W.generate(w, DEV)
+    rep = _check_workload(w, x)
+    print(w.name, rep)
+
+
+@pytest.mark.parametrize("idx", [1, 2, 3, 4])
+def test_workload_full_size_sampled(idx):
+    """Full-size launch (the configuration the benchmark times); the oracle checks sampled windows."""
+    w = W.WORKLOADS[idx]
+    x = W.generate(w, DEV)
+    per = 16 if idx >= 3 else 32
+    mid = (w.N // 2 // 64) * 64 + 7
+    sample = np.r_[0:per, mid:mid + per, w.N - per:w.N]
+    rep = _check_workload(w, x, sample=torch.from_numpy(sample).to(DEV))
+    print(w.name, rep)
+
+
+# ------------------------------------------------------------------------------------ edge cases
+
+
+def _random_inputs(N, K, V, dtype, seed, sigma=0.7, scale=2.0):
+    g = torch.Generator(device=DEV).manual_seed(seed)
+    t = (torch.randn((N, K, V), generator=g, device=DEV) * scale)
+    d = t + sigma * torch.randn((N, K, V), generator=g, device=DEV)
+    x = {"target_logits": t.to(dtype), "draft_logits": d.to(dtype),
+         "draft_tokens": torch.randint(0, V, (N, K), generator=g, device=DEV, dtype=torch.int32),
+         "uniforms": torch.rand((N, K), generator=g, device=DEV), "valid_len": None}
+    return x
+
+
+def _both_modes(x, c=0.05, temperature=1.0, eta=1.0, eps=0.5, ref_logp=None):
+    for mode in ("greedy", "stochastic"):
+        gpu = run_gpu(x, mode, c, temperature, eta, eps, ref_logp)
+        ref = run_oracle(x, mode, c, temperature, eta, eps, ref_logp)
+        compare_scores(gpu, ref, mode, x["uniforms"], eps=eps)
+    return gpu, ref
+
+
+@pytest.mark.parametrize("N,K,V,dtype", [
+    (5, 1, 8, torch.bfloat16),          # smallest vector row
+    (3, 32, 64, torch.bfloat16),        # largest K
+    (7, 3, 1001, torch.bfloat16),       # odd V: scalar path, rows not 16-byte aligned
+    (7, 3, 1001, torch.float32),
+    (2, 2, 2, torch.float32),           # smallest vocabulary
+    (4, 5, 8 * 2333, torch.bfloat16),   # several tiles plus a ragged tail of units
+    (1, 8, 128256, torch.bfloat16),     # few rows, large V: rows are split into segments
+    (3, 4, 50000, torch.float32),
+])
+def test_shapes_and_paths(N, K, V, dtype):
+    x = _random_inputs(N, K, V, dtype, seed=N * 1000 + K * 10 + V % 7)
+    _both_modes(x, temperature=0.9)
+
+
+def test_ragged_lengths_including_empty_windows():
+    N, K, V = 40, 10, 4096
+    x = _random_inputs(N, K, V, torch.bfloat16, seed=5)
+    x["valid_len"] = torch.randint(0, K + 1, (N,), device=DEV, dtype=torch.int32)
+    x["valid_len"][:3] = 0
+    x["valid_len"][3] = K
+    # poison the masked positions: they must be neither read into results nor scored
+    for n in range(N):
+        L = int(x["valid_len"][n])
+        x["draft_tokens"][n, L:] = -7
+    gpu, ref = _both_modes(x, eps=20.0)
+    assert B.ppow_read_error_flags(gpu["_workspace"]) == 0        # masked tokens are not looked at
+    for name in list(B.POSITION_OUTPUTS) + list(B.WINDOW_OUTPUTS):
+        assert float(gpu[name][:3].float().abs().sum()) == 0.0     # empty windows: all outputs 0
+
+
+def test_unaligned_base_pointer_takes_scalar_path():
+    N, K, V = 3, 2, 512
+    x = _random_inputs(N, K, V, torch.bfloat16, seed=6)
+    for key in ("target_logits", "draft_logits"):
+        flat = torch.empty(N * K * V + 1, dtype=torch.bfloat16, device=DEV)
+        flat[1:].copy_(x[key].flatten())
+        x[key] = flat[1:].view(N, K, V)                            # 2-byte aligned only
+        assert x[key].data_ptr() % 16 != 0
+    _both_modes(x)
+
+
+def test_argmax_ties_take_lowest_index():
+    N, K, V = 4, 3, 4096
+    x = _random_inputs(N, K, V, torch.bfloat16, seed=7)
+    t = x["target_logits"]
+    top = t.float().amax(-1, keepdim=True) + 1.0
+    idx = torch.tensor([4095, 17, 2048, 16, 3000], device=DEV)
+    t[:, :, idx] = top.to(torch.bfloat16)                          # five exact ties for the maximum
+    x["draft_tokens"][:, 0] = 16
+    x["draft_tokens"][:, 1] = 17
+    gpu, ref = _both_modes(x)
+    assert bool((gpu["target_argmax"] == 16).all())
+    g = run_gpu(x, "greedy", 0.05)
+    assert bool((g["accept_flag"][:, 0] == 1).all()) and bool((g["accept_flag"][:, 1] == 0).all())
+    # -0.0 and +0.0 tie
+    z = torch.full((1, 1, 64), -3.0, device=DEV, dtype=torch.bfloat16)
+    z[0, 0, 40] = 0.0
+    z[0, 0, 9] = -0.0
+    xz = {"target_logits": z, "draft_logits": z.clone(), "draft_tokens": torch.tensor([[9]], device=DEV, dtype=torch.int32),
+          "uniforms": torch.zeros((1, 1), device=DEV), "valid_len": None}
+    gz, rz = _both_modes(xz)
+    assert int(gz["target_argmax"][0, 0]) == 9 == int(rz["target_argmax"][0, 0])
+
+
+def test_identical_logits_zero_divergence_full_acceptance():
+    x = _random_inputs(6, 8, 32000, torch.bfloat16, seed=8)
+    x["draft_logits"] = x["target_logits"].clone()
+    gpu = run_gpu(x, "stochastic", 0.04)
+    assert float(gpu["kl"].abs().max()) == 0.0 and float(gpu["score"].abs().max()) == 0.0
+    assert bool((gpu["accepted_len"] == 8).all())
+    t = x["target_logits"].float()
+    first_max = torch.where(t == t.amax(-1, keepdim=True), torch.arange(t.shape[-1], device=DEV), t.shape[-1]).amin(-1)
+    x["draft_tokens"] = first_max.to(torch.int32)                  # lowest index among tied maxima
+    gpu = run_gpu(x, "greedy", 0.04)
+    assert bool((gpu["accepted_len"] == 8).all()) and float(gpu["delta"].abs().max()) == 0.0
+    _both_modes(x)
+
+
+def test_out_of_range_tokens_are_rejected_and_flagged():
+    x = _random_inputs(4, 4, 800, torch.bfloat16, seed=9)
+    x["draft_tokens"][1, 2] = 800
+    x["draft_tokens"][2, 0] = -1
+    gpu, ref = _both_modes(x)
+    assert B.ppow_read_error_flags(gpu["_workspace"]) & B.PPOW_FLAG_TOKEN_RANGE
+    assert int(gpu["accept_flag"][1, 2]) == 0 and int(gpu["accepted_len"][2]) == 0
+    assert float(gpu["logp_tok"][1, 2]) == float("-inf")
+
+
+def test_extreme_rows_exercise_reference_rebasing():
+    N, K, V = 4, 4, 8 * 1024
+    g = torch.Generator(device=DEV).manual_seed(10)
+    # steadily rising rows: almost every tile raises the running reference by far more than 2^64
+    ramp = torch.arange(V, device=DEV, dtype=torch.float32) * 0.9
+    t = ramp.view(1, 1, V) + torch.randn((N, K, V), generator=g, device=DEV)
+    d = ramp.flip(0).view(1, 1, V) * 0.5 + torch.randn((N, K, V), generator=g, device=DEV)
+    x = {"target_logits": t.to(torch.bfloat16), "draft_logits": d.to(torch.bfloat16),
+         "draft_tokens": torch.randint(0, V, (N, K), generator=g, device=DEV, dtype=torch.int32),
+         "uniforms": torch.rand((N, K), generator=g, device=DEV), "valid_len": None}
+    x["draft_tokens"][:, 0] = V - 1
+    _both_modes(x)
+    # Student-t spikes on both sides, float32 storage
+    spikes = torch.distributions.StudentT(3.0).sample((N, K, V)).to(DEV) * 400.0
+    x["target_logits"] = spikes.float()
+    x["draft_logits"] = (spikes + torch.distributions.StudentT(3.0).sample((N, K, V)).to(DEV) * 200.0).float()
+    _both_modes(x)
+
+
+def test_reference_window_logprob_variant_of_delta():
+    x = _random_inputs(9, 5, 2048, torch.bfloat16, seed=11, sigma=0.2)
+    ref_logp = -torch.rand(9, device=DEV) * 3.0
+    gpu, ref = _both_modes(x, eps=30.0, eta=0.7, ref_logp=ref_logp)
+    assert float(gpu["reward_dist"].max()) in (0.0, pytest.approx(0.7))
+
+
+def test_temperature_and_cost_parameters():
+    x = _random_inputs(6, 6, 4000, torch.bfloat16, seed=12)
+    for T, c in ((0.5, 0.0), (0.7, 0.12), (3.0, 1.5)):
+        _both_modes(x, c=c, temperature=T)
+
+
+def test_optional_outputs_may_be_omitted():
+    x = _random_inputs(4, 4, 1024, torch.bfloat16, seed=13)
+    p = B.make_params(4, 4, 1024, B.PPOW_BF16, B.PPOW_GREEDY, 0.05)
+    ws = B.alloc_workspace(B.ppow_score_workspace_bytes(p), DEV)
+    out = {"accepted_len": torch.full((4,), -1, device=DEV, dtype=torch.int32),
+           "score": torch.zeros(4, device=DEV)}
+    B.ppow_score_windows(p, x["draft_logits"], x["target_logits"], x["draft_tokens"], None, None, None, out, ws)
+    torch.cuda.synchronize()
+    full = run_gpu(x, "greedy", 0.05)
+    assert torch.equal(out["accepted_len"], full["accepted_len"]) and torch.equal(out["score"], full["score"])
+
+
+# ------------------------------------------------------------------------------------ selection
+
+
+@pytest.mark.parametrize("N,n_keep", [(1, 1), (2, 1), (64, 16), (1000, 1000), (4096, 410), (8192, 1639), (16384, 3),
+                                      (16385, 100), (70000, 14000), (3000, 0)])
+def test_selection_bit_exact_with_ties(N, n_keep):
+    g = torch.Generator(device=DEV).manual_seed(N + n_keep)
+    s = torch.rand(N, generator=g, device=DEV)
+    tie = torch.randint(0, N, (N // 3 + 1,), generator=g, device=DEV)
+    s[tie] = 0.5                                                    # many exact ties, some at the cut
+    s[torch.randint(0, N, (3,), generator=g, device=DEV)] = 0.0
+    s[torch.randint(0, N, (3,), generator=g, device=DEV)] = -0.0
+    compare_selection(s, n_keep)
+    compare_selection(torch.full((N,), 2.5, device=DEV), n_keep)    # all equal: the first n_keep indices
+    compare_selection(-s, n_keep)                                   # negative scores order correctly
+
+
+def test_status_codes_for_bad_arguments():
+    x = _random_inputs(2, 2, 64, torch.bfloat16, seed=14)
+    p = B.make_params(2, 2, 64, B.PPOW_BF16, B.PPOW_STOCHASTIC, 0.05)
+    ws = B.alloc_workspace(B.ppow_score_workspace_bytes(p), DEV)
+    out = B.alloc_outputs(2, 2, DEV)
+
+    def status(params=p, uniforms=x["uniforms"], outputs=out, workspace=ws):
+        try:
+            B.ppow_score_windows(params, x["draft_logits"], x["target_logits"], x["draft_tokens"], uniforms, None,
+                                 None, outputs, workspace)
+        except B.PpowError as e:
+            return e.status
+        return B.PPOW_OK
+
+    assert status() == B.PPOW_OK
+    assert status(uniforms=None) == B.PPOW_ERR_INVALID_ARG                      # stochastic needs uniforms
+    assert status(params=B.make_params(2, 2, 64, B.PPOW_BF16, 1, 0.05, temperature=0.0)) == B.PPOW_ERR_INVALID_ARG
+    assert status(params=B.make_params(2, 2, 1, B.PPOW_BF16, 1, 0.05)) == B.PPOW_ERR_INVALID_ARG
+    assert status(params=B.make_params(2, 33, 64, B.PPOW_BF16, 1, 0.05)) == B.PPOW_ERR_UNSUPPORTED
+    assert status(params=B.make_params(2, 2, 64, B.PPOW_BF16, 1, -1.0)) == B.PPOW_ERR_INVALID_ARG
+    assert status(workspace=ws[:16]) == B.PPOW_ERR_WORKSPACE
+    assert status(workspace=ws[1:]) == B.PPOW_ERR_WORKSPACE                     # misaligned
+    assert status(outputs={}) == B.PPOW_ERR_INVALID_ARG                         # accepted_len is required
+    assert status(params=B.make_params(0, 2, 64, B.PPOW_BF16, 1, 0.05)) == B.PPOW_OK   # N = 0: no-op
+    torch.cuda.synchronize()
+    s = torch.rand(10, device=DEV)
+    with pytest.raises(B.PpowError):
+        B.select_windows(s, 11)
+
+
+def test_host_buffer_entry_point_matches_device_path_with_chunking():
+    w = W.scaled(W.WORKLOADS[3], 70)
+    w = dataclasses.replace(w, V=4096)
+    x = W.generate(w, DEV)
+    dev_out = run_gpu(x, "stochastic", w.c, w.temperature)
+    dev_sel = B.select_windows(dev_out["score"], w.n_keep)
+    params = B.make_params(w.N, w.K, w.V, B.PPOW_BF16, B.PPOW_STOCHASTIC, w.c, w.temperature)
+    host = {k: (None if v is None else v.cpu().pin_memory()) for k, v in x.items()}
+    for chunk in (w.N, 16, 1):                                       # one chunk, several, one window at a time
+        out_host = {k: torch.zeros(v.shape, dtype=v.dtype).pin_memory() for k, v in dev_out.items() if not k.startswith("_")}
+        sel_host = torch.zeros((w.n_keep,), dtype=torch.int32).pin_memory()
+        mask_host = torch.zeros((w.N,), dtype=torch.uint8).pin_memory()
+        scratch = B.alloc_workspace(B.ppow_host_scratch_bytes(params, chunk), DEV)
+        B.ppow_score_and_select_host(params, host["draft_logits"], host["target_logits"], host["draft_tokens"],
+                                     host["uniforms"], host["valid_len"], None, out_host, w.n_keep, sel_host, mask_host,
+                                     scratch)
+        torch.cuda.synchronize()
+        for k, v in out_host.items():
+            assert torch.equal(v, dev_out[k].cpu()), (chunk, k)
+        assert torch.equal(sel_host, dev_sel.cpu())
+        assert int(mask_host.sum()) == w.n_keep
+    with pytest.raises(B.PpowError):
+        B.ppow_score_and_select_host(params, host["draft_logits"], host["target_logits"], host["draft_tokens"],
+                                     host["uniforms"], host["valid_len"], None, out_host, w.n_keep, sel_host, None,
+                                     B.alloc_workspace(1024, DEV))
