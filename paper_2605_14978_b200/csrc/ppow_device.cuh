@@ -169,9 +169,8 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
-// Reduce a warp's accumulators to one partial (valid in every lane).
-// `arg` is the thread's lowest vocabulary index holding its max_a (INT32_MAX if it saw nothing).
-__device__ __forceinline__ RowPartial warp_reduce(RowAcc acc, int32_t arg)
+// Reduce a warp's accumulators to one partial (valid in every lane); argmax is left unset.
+__device__ __forceinline__ RowPartial warp_reduce(RowAcc acc)
 {
     acc.fold();
     const float Ra = warp_max(acc.rho_a);
@@ -187,12 +186,8 @@ __device__ __forceinline__ RowPartial warp_reduce(RowAcc acc, int32_t arg)
     p.pad[0] = p.pad[1] = 0;
     p.E = warp_sum(acc.E[0]);
     p.D = warp_sum(acc.D[0]);
-    const float m = warp_max(acc.max_a);
-    int32_t idx = (acc.max_a == m) ? arg : INT32_MAX;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) idx = min(idx, __shfl_xor_sync(0xffffffffu, idx, o));
-    p.max_a = m;
-    p.argmax = idx;
+    p.max_a = warp_max(acc.max_a);
+    p.argmax = INT32_MAX;
     return p;
 }
 

@@ -52,25 +52,43 @@ __device__ __forceinline__ uint32_t fetch_item(const RowJob &job)
     return it;
 }
 
-// Block-level merge of per-warp partials; result written by thread 0.
-__device__ __forceinline__ void block_merge_and_store(const RowPartial &wp, RowPartial *smem_parts,
-                                                      RowPartial *dst)
+// End of a work item: merge the CTA's accumulators into one RowPartial and store it.
+// The vocabulary index of the row maximum is resolved only by the threads that hold that maximum
+// (usually one), between the two phases below.  Two barriers per item; the shared buffers may be
+// reused right after finish_end().
+struct ItemSmem {
+    RowPartial parts[ROW_WARPS];
+    int32_t arg;
+    uint32_t item[2];
+};
+
+// Phase 1: per-warp reduction into shared memory; returns the row (segment) maximum of the target.
+__device__ __forceinline__ float finish_begin(const RowAcc &acc, ItemSmem &sm)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (lane == 0) smem_parts[warp] = wp;
+    const RowPartial wp = warp_reduce(acc);
+    if (lane == 0) sm.parts[warp] = wp;
+    if (threadIdx.x == 0) sm.arg = INT32_MAX;
     __syncthreads();
+    float row_max = sm.parts[0].max_a;
+#pragma unroll
+    for (int w = 1; w < ROW_WARPS; ++w) row_max = fmaxf(row_max, sm.parts[w].max_a);
+    return row_max;
+}
+
+// Phase 2 (after the holders of the maximum have done atomicMin(&sm.arg, index)): merge and store.
+__device__ __forceinline__ void finish_end(ItemSmem &sm, RowPartial *dst)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (warp == 0) {
-        RowAcc acc;
-        int32_t arg = INT32_MAX;
-        if (lane < ROW_WARPS) {
-            acc = acc_from_partial(smem_parts[lane]);
-            arg = smem_parts[lane].argmax;
-        } else {
-            acc.reset();
-        }
-        RowPartial p = warp_reduce(acc, arg);
-        if (lane == 0) *dst = p;
+        RowAcc m;
+        if (lane < ROW_WARPS) m = acc_from_partial(sm.parts[lane]);
+        else m.reset();
+        const RowPartial p = warp_reduce(m);
+        if (lane == 0) *dst = p;          // argmax is patched in below
     }
+    __syncthreads();
+    if (threadIdx.x == 0) dst->argmax = sm.arg;
 }
 
 // ---- bf16, 16-byte vector path -----------------------------------------------------------------
@@ -113,18 +131,17 @@ __device__ __forceinline__ void bf16_group(const uint4 *__restrict__ pa, const u
 
 __global__ void __launch_bounds__(ROW_THREADS, 4) row_reduce_bf16_vec_kernel(const RowJob job)
 {
-    __shared__ RowPartial s_parts[ROW_WARPS];
-    __shared__ uint32_t s_item[2];
+    __shared__ ItemSmem sm;
 
     const int tid = threadIdx.x;
     const int32_t units_per_row = job.V >> 3;
-    if (tid == 0) s_item[0] = fetch_item(job);
+    if (tid == 0) sm.item[0] = fetch_item(job);
     __syncthreads();
-    uint32_t item = s_item[0];
+    uint32_t item = sm.item[0];
     int buf = 0;
 
     while (item < job.total_items) {
-        if (tid == 0) s_item[buf ^ 1] = fetch_item(job);   // prefetch the next item
+        if (tid == 0) sm.item[buf ^ 1] = fetch_item(job);   // prefetch the next item
 
         const uint32_t row = item / (uint32_t)job.segments;
         const int32_t seg = (int32_t)(item % (uint32_t)job.segments);
@@ -141,25 +158,27 @@ __global__ void __launch_bounds__(ROW_THREADS, 4) row_reduce_bf16_vec_kernel(con
         for (; u < u1; u += ROW_THREADS)
             bf16_group<1>(pa, pb, u, acc, job.s);
 
-        // lowest vocabulary index of this thread's maximum: rescan the group that raised it
-        int32_t arg = INT32_MAX;
-        if (acc.max_a > -INFINITY) {
-            const int32_t bu = acc.best >> 3, bn = acc.best & 7;
+        const float my_max = acc.max_a;
+        const int32_t my_best = acc.best;
+        const float row_max = finish_begin(acc, sm);
+        if (my_max == row_max) {
+            // lowest vocabulary index of this thread's maximum: re-read the group that raised it
+            const int32_t bu = my_best >> 3, bn = my_best & 7;
+            int32_t arg = INT32_MAX;
             for (int j = 0; j < bn && arg == INT32_MAX; ++j) {
-                const uint4 w4 = __ldg(pa + bu + j * ROW_THREADS);
+                const uint4 w4 = __ldcs(pa + bu + j * ROW_THREADS);
                 const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
                 for (int q = 3; q >= 0; --q) {
-                    if (bf16_hi(w[q]) == acc.max_a) arg = (bu + j * ROW_THREADS) * 8 + 2 * q + 1;
-                    if (bf16_lo(w[q]) == acc.max_a) arg = (bu + j * ROW_THREADS) * 8 + 2 * q;
+                    if (bf16_hi(w[q]) == my_max) arg = (bu + j * ROW_THREADS) * 8 + 2 * q + 1;
+                    if (bf16_lo(w[q]) == my_max) arg = (bu + j * ROW_THREADS) * 8 + 2 * q;
                 }
             }
+            atomicMin(&sm.arg, arg);
         }
-        const RowPartial wp = warp_reduce(acc, arg);
-        block_merge_and_store(wp, s_parts, job.partials + item);
-        __syncthreads();   // s_parts and s_item[buf^1] are stable past this point
+        finish_end(sm, job.partials + item);
         buf ^= 1;
-        item = s_item[buf];
+        item = sm.item[buf];
     }
 }
 
@@ -178,17 +197,16 @@ __device__ __forceinline__ float load_logit<uint16_t>(const uint16_t *p, size_t 
 template <typename T>
 __global__ void __launch_bounds__(ROW_THREADS, 4) row_reduce_generic_kernel(const RowJob job)
 {
-    __shared__ RowPartial s_parts[ROW_WARPS];
-    __shared__ uint32_t s_item[2];
+    __shared__ ItemSmem sm;
 
     const int tid = threadIdx.x;
-    if (tid == 0) s_item[0] = fetch_item(job);
+    if (tid == 0) sm.item[0] = fetch_item(job);
     __syncthreads();
-    uint32_t item = s_item[0];
+    uint32_t item = sm.item[0];
     int buf = 0;
 
     while (item < job.total_items) {
-        if (tid == 0) s_item[buf ^ 1] = fetch_item(job);
+        if (tid == 0) sm.item[buf ^ 1] = fetch_item(job);
 
         const uint32_t row = item / (uint32_t)job.segments;
         const int32_t seg = (int32_t)(item % (uint32_t)job.segments);
@@ -207,11 +225,12 @@ __global__ void __launch_bounds__(ROW_THREADS, 4) row_reduce_generic_kernel(cons
             acc.add_pair(a, b, job.s, 0);
             acc.flush();
         }
-        const RowPartial wp = warp_reduce(acc, arg);
-        block_merge_and_store(wp, s_parts, job.partials + item);
-        __syncthreads();
+        const float my_max = acc.max_a;
+        const float row_max = finish_begin(acc, sm);
+        if (my_max == row_max) atomicMin(&sm.arg, arg);
+        finish_end(sm, job.partials + item);
         buf ^= 1;
-        item = s_item[buf];
+        item = sm.item[buf];
     }
 }
 
@@ -294,10 +313,10 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
         double C = 1.0 - H / log((double)job.V);
         C = fmin(1.0, fmax(0.0, C));
         crit = C * KL;
-        const double lmax = (((double)mx * s - Ra) - l2Sa) * LN2;
+        const double lmax2 = fma((double)mx, s, -Ra) - l2Sa;   // log2 P(argmax); explicit fma: same rounding as lp2
 
         const int32_t tok = __ldg(job.tokens + row);
-        double lq;
+        double lq, lp2 = -INFINITY;
         if (tok < 0 || tok >= job.V) {
             atomicOr(&job.header->error_flags, (unsigned)PPOW_FLAG_TOKEN_RANGE);
             lp = -INFINITY;
@@ -306,8 +325,9 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
         } else {
             const double a_tok = raw_logit(job.target, job.dtype, row * job.V + tok);
             const double b_tok = raw_logit(job.draft, job.dtype, row * job.V + tok);
-            lp = ((a_tok * s - Ra) - l2Sa) * LN2;
-            lq = ((b_tok * s - Rb) - l2Sb) * LN2;
+            lp2 = fma(a_tok, s, -Ra) - l2Sa;
+            lp = lp2 * LN2;
+            lq = (fma(b_tok, s, -Rb) - l2Sb) * LN2;
             if (job.mode == PPOW_GREEDY) {
                 flag = (tok == arg);
             } else {
@@ -315,7 +335,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
                 flag = ((double)__ldg(job.uniforms + row) <= alpha);
             }
         }
-        gap = lmax - lp;
+        gap = (lmax2 - lp2) * LN2;   // differenced before scaling: exactly 0 when the token is the argmax
         o_kl = (float)KL; o_conf = (float)C; o_crit = (float)crit; o_lp = (float)lp; o_lq = (float)lq;
         o_arg = arg;
     }
