@@ -127,6 +127,30 @@ ppow_status ppow_score_windows_traced(const ppow_params *params,
                                       void *workspace, size_t workspace_bytes, void *cuda_stream,
                                       void *event_reduce_begin, void *event_reduce_end);
 
+/*
+ * ppow_score_windows without a workspace argument.  (An addition of this library; the paper has
+ * no counterpart.)  For callers that cannot obtain device scratch memory: code that runs beside a
+ * framework which already owns all device memory and whose allocator it cannot reach, or code
+ * that must not allocate after start-up.  The scratch is a fixed array of
+ * ppow_noalloc_scratch_bytes() (2 MiB) of device global memory inside the library image; every GPU
+ * that loads the library holds it until the process exits.  Inputs, outputs, stream and results
+ * are exactly those of ppow_score_windows.  No memory is allocated or freed by this call.
+ *   - Returns PPOW_ERR_UNSUPPORTED, launching nothing, when
+ *     ppow_score_workspace_bytes(params) > ppow_noalloc_scratch_bytes().
+ *   - All calls on one device share the array, and it keeps the previous call's contents; the work
+ *     counter and error word that must start at zero are cleared on the stream by every call.
+ *     Calls that overlap on the GPU (other streams or host threads) race on it: serialise them.
+ *   - The first call on each device looks up the array's device address, which may load the
+ *     module: make that first call outside any stream capture.
+ *   - The error word of this call cannot be read back with ppow_read_error_flags.
+ */
+size_t ppow_noalloc_scratch_bytes(void);
+ppow_status ppow_score_windows_noalloc(const ppow_params *params,
+                                       const void *draft_logits, const void *target_logits,
+                                       const int32_t *draft_tokens, const float *uniforms,
+                                       const int32_t *valid_len, const float *ref_logp,
+                                       const ppow_outputs *out, void *cuda_stream);
+
 /* Copies the error word that the last ppow_score_windows call on `workspace` left behind into
  * *flags_host (PPOW_FLAG_* bits) and synchronises `cuda_stream` to do so.  Returns
  * PPOW_ERR_DEVICE_TIMEOUT if that bit is set, PPOW_ERR_CUDA on a CUDA failure, else PPOW_OK. */

@@ -23,7 +23,8 @@ PPOW_FLAG_TOKEN_RANGE, PPOW_FLAG_DEVICE_TIMEOUT = 1, 2
 
 EXPORTS = ("ppow_score_workspace_bytes", "ppow_score_windows", "ppow_score_windows_traced", "ppow_read_error_flags",
            "ppow_select_workspace_bytes", "ppow_select_windows", "ppow_host_scratch_bytes",
-           "ppow_score_and_select_host", "ppow_status_string", "ppow_version")
+           "ppow_score_and_select_host", "ppow_noalloc_scratch_bytes", "ppow_score_windows_noalloc",
+           "ppow_status_string", "ppow_version")
 
 POSITION_OUTPUTS = {"accept_flag": torch.uint8, "kl": torch.float32, "conf": torch.float32, "crit": torch.float32,
                     "logp_tok": torch.float32, "logq_tok": torch.float32, "target_argmax": torch.int32}
@@ -82,6 +83,11 @@ def load_library():
     lib.ppow_score_and_select_host.restype = ctypes.c_int
     lib.ppow_score_and_select_host.argtypes = [ctypes.POINTER(ppow_params), vp, vp, vp, vp, vp, vp,
                                                ctypes.POINTER(ppow_outputs), i32, vp, vp, vp, sz, vp]
+    lib.ppow_noalloc_scratch_bytes.restype = sz
+    lib.ppow_noalloc_scratch_bytes.argtypes = []
+    lib.ppow_score_windows_noalloc.restype = ctypes.c_int
+    lib.ppow_score_windows_noalloc.argtypes = [ctypes.POINTER(ppow_params), vp, vp, vp, vp, vp, vp,
+                                               ctypes.POINTER(ppow_outputs), vp]
     lib.ppow_status_string.restype = ctypes.c_char_p
     lib.ppow_status_string.argtypes = [ctypes.c_int]
     lib.ppow_version.restype = ctypes.c_int
@@ -202,6 +208,32 @@ def ppow_select_windows(score, n_keep: int, selected, mask, workspace, stream=No
         workspace.numel() if workspace is not None else 0, _stream_ptr(stream))
     if st != PPOW_OK:
         raise PpowError(st, "ppow_select_windows")
+
+
+def ppow_noalloc_scratch_bytes() -> int:
+    return int(load_library().ppow_noalloc_scratch_bytes())
+
+
+def ppow_score_windows_noalloc(params: ppow_params, draft_logits, target_logits, draft_tokens, uniforms, valid_len,
+                               ref_logp, outputs: dict, stream=None) -> None:
+    """ppow_score_windows for callers that cannot hand over a workspace: the library's built-in 2 MiB
+    scratch array is used instead.  The binding itself allocates nothing here; ``outputs`` must hold
+    preallocated CUDA tensors.  Calls on one device must not overlap (they share the array)."""
+    lib = load_library()
+    lt = torch.float32 if params.dtype == PPOW_F32 else torch.bfloat16
+    o = ppow_outputs()
+    for name, _ in ppow_outputs._fields_:
+        want = POSITION_OUTPUTS.get(name) or WINDOW_OUTPUTS.get(name)
+        p = _dev_ptr(outputs.get(name), want, name)
+        setattr(o, name, p.value if p is not None else None)
+    st = lib.ppow_score_windows_noalloc(
+        ctypes.byref(params),
+        _dev_ptr(draft_logits, lt, "draft_logits"), _dev_ptr(target_logits, lt, "target_logits"),
+        _dev_ptr(draft_tokens, torch.int32, "draft_tokens"), _dev_ptr(uniforms, torch.float32, "uniforms"),
+        _dev_ptr(valid_len, torch.int32, "valid_len"), _dev_ptr(ref_logp, torch.float32, "ref_logp"),
+        ctypes.byref(o), _stream_ptr(stream))
+    if st != PPOW_OK:
+        raise PpowError(st, "ppow_score_windows_noalloc")
 
 
 def _host_ptr(t: Optional[torch.Tensor], dtype=None, name="tensor"):
