@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ppow", choices=["ppow", "reference"])
     ap.add_argument("--workload", default="llama3_like", choices=[w.name for w in W.WORKLOADS])
@@ -205,6 +205,7 @@ def run_reference(args):
 def run_ppow(args):
     from paper_2605_14978_b200 import binding as B
     from paper_2605_14978_b200 import build as build_mod
+    from paper_2605_14978_b200 import sharding as S
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py --impl ppow needs a CUDA device; there is no CPU path")
@@ -231,7 +232,6 @@ def run_ppow(args):
     params = B.make_params(N, K, V, B.PPOW_F32 if w.dtype == "f32" else B.PPOW_BF16, bmode, w.c, w.temperature)
     out = B.alloc_outputs(N, K, dev)
     ws = B.alloc_workspace(B.ppow_score_workspace_bytes(params), dev)
-    all_scores = torch.empty((n_total,), dtype=torch.float32, device=dev) if world > 1 else out["score"]
     selected = torch.empty((n_keep,), dtype=torch.int32, device=dev)
     sel_ws = B.alloc_workspace(B.ppow_select_workspace_bytes(n_total), dev)
     stream = torch.cuda.current_stream()
@@ -239,10 +239,8 @@ def run_ppow(args):
     def step(ev0=None, ev1=None):
         B.ppow_score_windows_traced(params, x["draft_logits"], x["target_logits"], x["draft_tokens"], x["uniforms"],
                                     x["valid_len"], None, out, ws, stream, ev0, ev1)
-        if world > 1:
-            import torch.distributed as dist
-            dist.all_gather_into_tensor(all_scores, out["score"])       # the one exchange step of the path
-        B.ppow_select_windows(all_scores, n_keep, selected, None, sel_ws, stream)
+        scores = S.gather_scores(out["score"], n_total) if world > 1 else out["score"]   # the one exchange step
+        B.ppow_select_windows(scores, n_keep, selected, None, sel_ws, stream)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -311,7 +309,7 @@ def run_ppow(args):
         import oracle
         oracle.build()
         cores = os.cpu_count() or 1
-        n_sample_chunks = min(n_chunks, 8)
+        n_sample_chunks = min(n_chunks, 16)     # ~25 core-seconds of oracle work on the headline workload
         idx = slice(0, min(N, n_sample_chunks * W.CHUNK))
         xs = {k: (None if v is None else v[idx].cpu()) for k, v in x.items()}
         dt = time_oracle(w, mode, xs, cores)
