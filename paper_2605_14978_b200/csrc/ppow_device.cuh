@@ -27,10 +27,9 @@ struct __align__(16) RowPartial {
     float rho_a, rho_b;   // references, log2 units
     float Sa, Sb;         // sums relative to those references (leading parts)
     float Sa_lo, Sb_lo;   // their compensation terms: the sums are Sa + Sa_lo, Sb + Sb_lo
-    float E, D;
+    double E, D;          // weighted sums relative to the same references
     float max_a;          // largest stored target logit seen
     int32_t argmax;       // its lowest vocabulary index
-    int32_t pad[2];
 };
 static_assert(sizeof(RowPartial) == 48, "RowPartial layout");
 
@@ -53,37 +52,48 @@ __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w 
 
 // Per-thread running state for one row (or row segment).
 //
-// Sa and Sb are what log-probabilities are read from, and a confident distribution puts almost all
-// of a sum into one term: once an f32 accumulator holds that term, every later small term is rounded
-// at its ulp (6e-8 relative each, hundreds of times).  So both sums are kept as tile-local partials
-// (Sa[], Sb[], restarted from zero by flush()) that are folded into a running (hi, lo) pair with an
+// A confident distribution puts almost all of a sum into one term: once an f32 accumulator holds
+// that term, every later small term is rounded at its ulp (6e-8 relative each, thousands of times
+// when a lane walks a whole row).  So all four sums are kept as tile-local partials (Sa, Sb, E, D,
+// restarted from zero by flush()) that are folded into running (hi, lo) pairs with an
 // error-compensated add; only the few adds inside one tile can be absorbed.
+//
+// The tile-local accumulators are float2: lane .x takes the even vocabulary entries of a packed bf16
+// word, lane .y the odd ones, so that the arithmetic runs on sm_100's packed f32x2 instructions
+// (__ffma2_rn / __fadd2_rn: one issue slot for two IEEE fma/add operations).
 struct RowAcc {
     float rho_a, rho_b;
-    float Sa[2], Sb[2], E[2], D[2];
-    float Sa_hi, Sa_lo, Sb_hi, Sb_lo;
+    float2 Sa, Sb, E, D;
+    float Sa_hi, Sa_lo, Sb_hi, Sb_lo, E_hi, E_lo, D_hi, D_lo;
     float max_a;
     int32_t best;       // where max_a was first seen (meaning defined by the caller)
 
     __device__ __forceinline__ void reset()
     {
         rho_a = rho_b = RHO_INIT;
-        Sa[0] = Sa[1] = Sb[0] = Sb[1] = E[0] = E[1] = D[0] = D[1] = 0.0f;
-        Sa_hi = Sa_lo = Sb_hi = Sb_lo = 0.0f;
+        Sa = Sb = E = D = make_float2(0.0f, 0.0f);
+        Sa_hi = Sa_lo = Sb_hi = Sb_lo = E_hi = E_lo = D_hi = D_lo = 0.0f;
         max_a = -INFINITY;
         best = 0;
+    }
+
+    // hi + p -> (hi, lo += rounding error); p and hi of any sign (Knuth's two-sum).
+    static __device__ __forceinline__ void two_sum(float &hi, float &lo, float p)
+    {
+        const float t = hi + p;
+        const float bp = t - hi;
+        lo += (hi - (t - bp)) + (p - bp);
+        hi = t;
     }
 
     // Fold the tile-local partial sums into the compensated running sums (call once per tile).
     __device__ __forceinline__ void flush()
     {
-        const float pa = Sa[0] + Sa[1], pb = Sb[0] + Sb[1];
-        const float ta = Sa_hi + pa, tb = Sb_hi + pb;
-        Sa_lo += pa - (ta - Sa_hi);
-        Sb_lo += pb - (tb - Sb_hi);
-        Sa_hi = ta;
-        Sb_hi = tb;
-        Sa[0] = Sa[1] = Sb[0] = Sb[1] = 0.0f;
+        two_sum(Sa_hi, Sa_lo, Sa.x + Sa.y);
+        two_sum(Sb_hi, Sb_lo, Sb.x + Sb.y);
+        two_sum(E_hi, E_lo, E.x + E.y);
+        two_sum(D_hi, D_lo, D.x + D.y);
+        Sa = Sb = E = D = make_float2(0.0f, 0.0f);
     }
 
     // Move both references (log2 units).  Only between tiles (after flush()).  With x' = x - d,
@@ -93,11 +103,12 @@ struct RowAcc {
     __device__ __forceinline__ void rebase(float new_rho_a, float new_rho_b)
     {
         const float da = rho_a - new_rho_a, db = rho_b - new_rho_b;
+        if (da == 0.0f && db == 0.0f) return;
         const float fa = ex2_approx(da), fb = ex2_approx(db);
         const float S = Sa_hi + Sa_lo;
-        E[0] = fa * fmaf(da, S, E[0] + E[1]);
-        D[0] = fa * fmaf(da - db, S, D[0] + D[1]);
-        E[1] = D[1] = 0.0f;
+        E_hi = fa * fmaf(da, S, E_hi + E_lo);
+        D_hi = fa * fmaf(da - db, S, D_hi + D_lo);
+        E_lo = D_lo = 0.0f;
         Sa_hi *= fa;
         Sa_lo *= fa;
         Sb_hi *= fb;
@@ -106,24 +117,32 @@ struct RowAcc {
         rho_b = new_rho_b;
     }
 
-    // One (target, draft) pair already widened to f32.  i selects the accumulator set.
-    __device__ __forceinline__ void add_pair(float a, float b, float s, int i)
+    // One (target, draft) pair already widened to f32 (scalar path; accumulates into lane .x).
+    __device__ __forceinline__ void add_pair(float a, float b, float s)
     {
         const float xa = fmaf(a, s, -rho_a);
         const float xb = fmaf(b, s, -rho_b);
         const float ea = ex2_approx(xa);
         const float eb = ex2_approx(xb);
-        Sa[i] += ea;
-        Sb[i] += eb;
-        E[i] = fmaf(ea, xa, E[i]);
-        D[i] = fmaf(ea, xa - xb, D[i]);
+        Sa.x += ea;
+        Sb.x += eb;
+        E.x = fmaf(ea, xa, E.x);
+        D.x = fmaf(ea, xa - xb, D.x);
     }
 
-    // Two packed bf16 pairs.
-    __device__ __forceinline__ void add_word(uint32_t wa, uint32_t wb, float s)
+    // Two packed bf16 pairs: the same operations as two add_pair calls, two per instruction.
+    // s2 = (s, s), nra = (-rho_a, -rho_a), nrb = (-rho_b, -rho_b).
+    __device__ __forceinline__ void add_word(uint32_t wa, uint32_t wb, float2 s2, float2 nra, float2 nrb)
     {
-        add_pair(bf16_lo(wa), bf16_lo(wb), s, 0);
-        add_pair(bf16_hi(wa), bf16_hi(wb), s, 1);
+        const float2 xa = __ffma2_rn(make_float2(bf16_lo(wa), bf16_hi(wa)), s2, nra);
+        const float2 xb = __ffma2_rn(make_float2(bf16_lo(wb), bf16_hi(wb)), s2, nrb);
+        const float2 ea = make_float2(ex2_approx(xa.x), ex2_approx(xa.y));
+        const float2 eb = make_float2(ex2_approx(xb.x), ex2_approx(xb.y));
+        Sa = __fadd2_rn(Sa, ea);
+        Sb = __fadd2_rn(Sb, eb);
+        E = __ffma2_rn(ea, xa, E);
+        const float2 dx = __ffma2_rn(xb, make_float2(-1.0f, -1.0f), xa);   // xa - xb, one rounding
+        D = __ffma2_rn(ea, dx, D);
     }
 
     // Raise the references if this tile's maxima (raw logit units) call for it.
@@ -132,12 +151,6 @@ struct RowAcc {
         const bool up_a = fmaf(tile_max_a, s, -rho_a) > REBASE_LOG2;
         const bool up_b = fmaf(tile_max_b, s, -rho_b) > REBASE_LOG2;
         if (up_a | up_b) rebase(up_a ? tile_max_a * s : rho_a, up_b ? tile_max_b * s : rho_b);
-    }
-
-    __device__ __forceinline__ void fold()
-    {
-        E[0] += E[1]; D[0] += D[1];
-        E[1] = D[1] = 0.0f;
     }
 };
 
@@ -169,10 +182,16 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
+__device__ __forceinline__ double warp_sum_f64(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
 // Reduce a warp's accumulators to one partial (valid in every lane); argmax is left unset.
 __device__ __forceinline__ RowPartial warp_reduce(RowAcc acc)
 {
-    acc.fold();
     const float Ra = warp_max(acc.rho_a);
     const float Rb = warp_max(acc.rho_b);
     acc.rebase(Ra, Rb);
@@ -183,22 +202,11 @@ __device__ __forceinline__ RowPartial warp_reduce(RowAcc acc)
     warp_sum_pair(acc.Sb_hi, acc.Sb_lo);
     p.Sa = acc.Sa_hi; p.Sa_lo = acc.Sa_lo;
     p.Sb = acc.Sb_hi; p.Sb_lo = acc.Sb_lo;
-    p.pad[0] = p.pad[1] = 0;
-    p.E = warp_sum(acc.E[0]);
-    p.D = warp_sum(acc.D[0]);
+    p.E = warp_sum_f64((double)acc.E_hi + (double)acc.E_lo);
+    p.D = warp_sum_f64((double)acc.D_hi + (double)acc.D_lo);
     p.max_a = warp_max(acc.max_a);
     p.argmax = INT32_MAX;
     return p;
-}
-
-__device__ __forceinline__ RowAcc acc_from_partial(const RowPartial &p)
-{
-    RowAcc a;
-    a.reset();
-    a.rho_a = p.rho_a; a.rho_b = p.rho_b;
-    a.Sa_hi = p.Sa; a.Sa_lo = p.Sa_lo; a.Sb_hi = p.Sb; a.Sb_lo = p.Sb_lo; a.E[0] = p.E; a.D[0] = p.D;
-    a.max_a = p.max_a;
-    return a;
 }
 
 }  // namespace ppow

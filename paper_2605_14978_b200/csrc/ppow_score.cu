@@ -2,14 +2,14 @@
 // and the host entry points ppow_score_windows / ppow_score_workspace_bytes / ppow_read_error_flags.
 #include "../../include/ppow.h"
 #include "ppow_device.cuh"
+#include "ppow_async.cuh"
 
 #include <math.h>
 
 namespace ppow {
 
-constexpr int ROW_THREADS = 256;   // threads per CTA in the row-reduction kernels
-constexpr int ROW_WARPS = ROW_THREADS / 32;
-constexpr int UNROLL = 4;          // 16-byte units per thread per tensor in flight
+constexpr int ROW_THREADS = 256;   // threads per CTA of the scalar row-reduction kernels
+constexpr int UNROLL = 4;          // 16-byte units per thread per tensor in flight (< 8: packed with the unit index)
 constexpr int MAX_SEGMENTS = 16;   // a row is split into at most this many work items
 constexpr size_t WS_HEADER_BYTES = 256;
 
@@ -52,133 +52,218 @@ __device__ __forceinline__ uint32_t fetch_item(const RowJob &job)
     return it;
 }
 
-// End of a work item: merge the CTA's accumulators into one RowPartial and store it.
-// The vocabulary index of the row maximum is resolved only by the threads that hold that maximum
-// (usually one), between the two phases below.  Two barriers per item; the shared buffers may be
-// reused right after finish_end().
-struct ItemSmem {
-    RowPartial parts[ROW_WARPS];
-    int32_t arg;
-    uint32_t item[2];
+constexpr uint32_t BF16X2_NEG_INF = 0xff80ff80u;   // packed bf16 (-inf, -inf): neutral for the tile maximum
+
+__device__ __forceinline__ int32_t warp_min_i32(int32_t v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = min(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// ---- bf16, bulk-copy pipeline, one warp per work item ----------------------------------------------
+// Each warp takes (row, segment) items from the work counter on its own; no block barrier is used after
+// set-up, so the warps of an SM drift apart.  The logits reach the warp through its own ring of
+// PIPE_STAGES shared-memory stages filled by bulk copies (cp.async.bulk + mbarrier): while the warp
+// computes on one tile, the copies of the next PIPE_STAGES - 1 tiles are in flight, across the end of
+// an item into the next one.  Loads never pause for the arithmetic, the end-of-item reduction or the
+// argmax re-read, and they hold no registers while in flight.
+#ifndef PIPE_WARPS
+#define PIPE_WARPS 8
+#endif
+#ifndef PIPE_STAGES
+#define PIPE_STAGES 3
+#endif
+#ifndef PIPE_MIN_CTAS
+#define PIPE_MIN_CTAS 2
+#endif
+constexpr int TILE_UNITS = 32 * UNROLL;       // 16-byte units per tile per tensor
+constexpr int TILE_BYTES = TILE_UNITS * 16;   // 2 KB per tensor
+constexpr int ITEM_RING = 8;                  // > PIPE_STAGES + 1 item ids between producer and consumer
+constexpr uint32_t WAIT_LIMIT = 1u << 20;     // probes of one mbarrier before the kernel gives up
+constexpr size_t PIPE_SMEM_BYTES = (size_t)PIPE_WARPS * PIPE_STAGES * 2 * TILE_BYTES;
+
+struct ItemCursor {
+    uint32_t item;          // >= total_items: nothing left
+    int32_t u, u1;          // next unit and end of the item, relative to the row
+    const uint4 *pa, *pb;   // row bases
 };
 
-// Phase 1: per-warp reduction into shared memory; returns the row (segment) maximum of the target.
-__device__ __forceinline__ float finish_begin(const RowAcc &acc, ItemSmem &sm)
+__device__ __forceinline__ void open_item(const RowJob &job, ItemCursor &c, uint32_t item)
 {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const RowPartial wp = warp_reduce(acc);
-    if (lane == 0) sm.parts[warp] = wp;
-    if (threadIdx.x == 0) sm.arg = INT32_MAX;
-    __syncthreads();
-    float row_max = sm.parts[0].max_a;
-#pragma unroll
-    for (int w = 1; w < ROW_WARPS; ++w) row_max = fmaxf(row_max, sm.parts[w].max_a);
-    return row_max;
+    c.item = item;
+    c.u = c.u1 = 0;
+    c.pa = c.pb = nullptr;
+    if (item >= job.total_items) return;
+    const int32_t units_per_row = job.V >> 3;
+    const uint32_t row = item / (uint32_t)job.segments;
+    const int32_t seg = (int32_t)(item % (uint32_t)job.segments);
+    c.u = (int32_t)(((int64_t)units_per_row * seg) / job.segments);
+    c.u1 = (int32_t)(((int64_t)units_per_row * (seg + 1)) / job.segments);
+    c.pa = reinterpret_cast<const uint4 *>(job.target) + (size_t)row * units_per_row;
+    c.pb = reinterpret_cast<const uint4 *>(job.draft) + (size_t)row * units_per_row;
 }
 
-// Phase 2 (after the holders of the maximum have done atomicMin(&sm.arg, index)): merge and store.
-__device__ __forceinline__ void finish_end(ItemSmem &sm, RowPartial *dst)
+// One tile out of shared memory.  `nu` = units of this lane that exist (UNROLL unless MASKED);
+// refill() is called once every value of the stage sits in registers.
+template <bool MASKED, typename Refill>
+__device__ __forceinline__ void pipe_tile(const uint4 *sa, const uint4 *sb, int32_t u, int nu, RowAcc &acc,
+                                          float s, Refill refill)
 {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (warp == 0) {
-        RowAcc m;
-        if (lane < ROW_WARPS) m = acc_from_partial(sm.parts[lane]);
-        else m.reset();
-        const RowPartial p = warp_reduce(m);
-        if (lane == 0) *dst = p;          // argmax is patched in below
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) dst->argmax = sm.arg;
-}
-
-// ---- bf16, 16-byte vector path -----------------------------------------------------------------
-// Requires V % 8 == 0 and 16-byte aligned tensors.  Each thread streams 16-byte units
-// u = u0 + tid + j*ROW_THREADS with UNROLL loads per tensor in flight; both tensors are read once.
-
-template <int NU>
-__device__ __forceinline__ void bf16_group(const uint4 *__restrict__ pa, const uint4 *__restrict__ pb,
-                                           int32_t u, RowAcc &acc, float s)
-{
-    uint4 A[NU], B[NU];
+    const int lane = threadIdx.x & 31;
+    uint4 A[UNROLL], B[UNROLL];
+    const uint4 none = make_uint4(BF16X2_NEG_INF, BF16X2_NEG_INF, BF16X2_NEG_INF, BF16X2_NEG_INF);
 #pragma unroll
-    for (int j = 0; j < NU; ++j) A[j] = __ldcs(pa + u + j * ROW_THREADS);
+    for (int j = 0; j < UNROLL; ++j) A[j] = (!MASKED || j < nu) ? sa[j * 32 + lane] : none;
 #pragma unroll
-    for (int j = 0; j < NU; ++j) B[j] = __ldcs(pb + u + j * ROW_THREADS);
+    for (int j = 0; j < UNROLL; ++j) B[j] = (!MASKED || j < nu) ? sb[j * 32 + lane] : none;
 
     uint32_t ma = max_bf16x2(max_bf16x2(A[0].x, A[0].y), max_bf16x2(A[0].z, A[0].w));
     uint32_t mb = max_bf16x2(max_bf16x2(B[0].x, B[0].y), max_bf16x2(B[0].z, B[0].w));
 #pragma unroll
-    for (int j = 1; j < NU; ++j) {
+    for (int j = 1; j < UNROLL; ++j) {
         ma = max_bf16x2(ma, max_bf16x2(max_bf16x2(A[j].x, A[j].y), max_bf16x2(A[j].z, A[j].w)));
         mb = max_bf16x2(mb, max_bf16x2(max_bf16x2(B[j].x, B[j].y), max_bf16x2(B[j].z, B[j].w)));
     }
     const float tmax_a = fmaxf(bf16_lo(ma), bf16_hi(ma));
     const float tmax_b = fmaxf(bf16_lo(mb), bf16_hi(mb));
     acc.guard(tmax_a, tmax_b, s);
-    if (tmax_a > acc.max_a) {   // strict: an equal value seen later has a higher index
+    if (tmax_a > acc.max_a) {
         acc.max_a = tmax_a;
-        acc.best = u * 8 + NU;  // unit index and group size packed: (u << 3) | NU, NU in {1, 4}
+        acc.best = u * 8 + nu;
     }
+    refill();   // the tile maxima consumed every word of the stage: it may be overwritten now
+    const float2 s2 = make_float2(s, s);
+    const float2 nra = make_float2(-acc.rho_a, -acc.rho_a), nrb = make_float2(-acc.rho_b, -acc.rho_b);
 #pragma unroll
-    for (int j = 0; j < NU; ++j) {
-        acc.add_word(A[j].x, B[j].x, s);
-        acc.add_word(A[j].y, B[j].y, s);
-        acc.add_word(A[j].z, B[j].z, s);
-        acc.add_word(A[j].w, B[j].w, s);
+    for (int j = 0; j < UNROLL; ++j) {
+        if (!MASKED || j < nu) {
+            acc.add_word(A[j].x, B[j].x, s2, nra, nrb);
+            acc.add_word(A[j].y, B[j].y, s2, nra, nrb);
+            acc.add_word(A[j].z, B[j].z, s2, nra, nrb);
+            acc.add_word(A[j].w, B[j].w, s2, nra, nrb);
+        }
     }
     acc.flush();
 }
 
-__global__ void __launch_bounds__(ROW_THREADS, 4) row_reduce_bf16_vec_kernel(const RowJob job)
+__global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_bf16_pipe_kernel(const RowJob job)
 {
-    __shared__ ItemSmem sm;
+    extern __shared__ __align__(128) unsigned char pipe_smem[];
+    __shared__ __align__(8) uint64_t full_bar[PIPE_WARPS][PIPE_STAGES];
+    __shared__ uint32_t item_ring[PIPE_WARPS][ITEM_RING];
 
-    const int tid = threadIdx.x;
-    const int32_t units_per_row = job.V >> 3;
-    if (tid == 0) sm.item[0] = fetch_item(job);
-    __syncthreads();
-    uint32_t item = sm.item[0];
-    int buf = 0;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned char *stages = pipe_smem + (size_t)warp * PIPE_STAGES * 2 * TILE_BYTES;
+    const uint32_t stages_addr = smem_addr(stages);
+    const uint32_t bars_addr = smem_addr(&full_bar[warp][0]);
 
-    while (item < job.total_items) {
-        if (tid == 0) sm.item[buf ^ 1] = fetch_item(job);   // prefetch the next item
-
-        const uint32_t row = item / (uint32_t)job.segments;
-        const int32_t seg = (int32_t)(item % (uint32_t)job.segments);
-        const int32_t u0 = (int32_t)(((int64_t)units_per_row * seg) / job.segments);
-        const int32_t u1 = (int32_t)(((int64_t)units_per_row * (seg + 1)) / job.segments);
-        const uint4 *pa = reinterpret_cast<const uint4 *>(job.target) + (size_t)row * units_per_row;
-        const uint4 *pb = reinterpret_cast<const uint4 *>(job.draft) + (size_t)row * units_per_row;
-
-        RowAcc acc;
-        acc.reset();
-        int32_t u = u0 + tid;
-        for (; u + (UNROLL - 1) * ROW_THREADS < u1; u += UNROLL * ROW_THREADS)
-            bf16_group<UNROLL>(pa, pb, u, acc, job.s);
-        for (; u < u1; u += ROW_THREADS)
-            bf16_group<1>(pa, pb, u, acc, job.s);
-
-        const float my_max = acc.max_a;
-        const int32_t my_best = acc.best;
-        const float row_max = finish_begin(acc, sm);
-        if (my_max == row_max) {
-            // lowest vocabulary index of this thread's maximum: re-read the group that raised it
-            const int32_t bu = my_best >> 3, bn = my_best & 7;
-            int32_t arg = INT32_MAX;
-            for (int j = 0; j < bn && arg == INT32_MAX; ++j) {
-                const uint4 w4 = __ldcs(pa + bu + j * ROW_THREADS);
-                const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+    if (lane == 0) {
 #pragma unroll
-                for (int q = 3; q >= 0; --q) {
-                    if (bf16_hi(w[q]) == my_max) arg = (bu + j * ROW_THREADS) * 8 + 2 * q + 1;
-                    if (bf16_lo(w[q]) == my_max) arg = (bu + j * ROW_THREADS) * 8 + 2 * q;
+        for (int st = 0; st < PIPE_STAGES; ++st) mbar_init(bars_addr + 8 * st, 1);
+        mbar_init_fence();
+    }
+    __syncthreads();
+
+    // Producer side: P walks the items this warp takes from the work counter and issues one tile per call.
+    ItemCursor P, C;
+    uint32_t produced = 0, consumed = 0;   // items opened by each side
+    uint32_t pending = 0;                   // stages with a copy in flight
+    uint32_t first = 0, upcoming = 0;       // `upcoming` (lane 0): id fetched ahead for the item after P's
+    if (lane == 0) first = fetch_item(job);
+    first = __shfl_sync(0xffffffffu, first, 0);
+    if (lane == 0) {
+        item_ring[warp][0] = first;
+        if (first < job.total_items) upcoming = fetch_item(job);
+    }
+    open_item(job, P, first);
+    open_item(job, C, first);
+    produced = consumed = 1;
+
+    auto produce = [&](int st) {
+        if (P.item >= job.total_items) return;
+        const int32_t n = min(TILE_UNITS, P.u1 - P.u);
+        if (lane == 0) {
+            const uint32_t bar = bars_addr + 8 * st, dst = stages_addr + st * 2 * TILE_BYTES;
+            mbar_arrive_expect_tx(bar, 2u * (uint32_t)n * 16u);
+            bulk_load(dst, P.pa + P.u, (uint32_t)n * 16u, bar);
+            bulk_load(dst + TILE_BYTES, P.pb + P.u, (uint32_t)n * 16u, bar);
+        }
+        pending |= 1u << st;
+        P.u += n;
+        if (P.u >= P.u1) {
+            const uint32_t nx = __shfl_sync(0xffffffffu, upcoming, 0);
+            if (lane == 0) {
+                item_ring[warp][produced % ITEM_RING] = nx;
+                if (nx < job.total_items) upcoming = fetch_item(job);
+            }
+            ++produced;
+            open_item(job, P, nx);
+        }
+    };
+
+#pragma unroll
+    for (int st = 0; st < PIPE_STAGES; ++st) produce(st);
+
+    uint32_t phases = 0;
+    int st = 0;
+    RowAcc acc;
+    acc.reset();
+    while (C.item < job.total_items) {
+        const int32_t n = min(TILE_UNITS, C.u1 - C.u);
+        // every lane waits (the tile becomes visible to the lanes that observed the phase); the vote keeps
+        // the warp together if the limit is hit by only some of them
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(bars_addr + 8 * st, (phases >> st) & 1u, WAIT_LIMIT))) {
+            // give up: report, wait (bounded) for the copies still aimed at this warp's stages, leave
+            if (lane == 0) atomicOr(&job.header->error_flags, (unsigned)PPOW_FLAG_DEVICE_TIMEOUT);
+#pragma unroll
+            for (int q = 0; q < PIPE_STAGES; ++q)
+                if (pending & (1u << q)) mbar_wait_bounded(bars_addr + 8 * q, (phases >> q) & 1u, WAIT_LIMIT);
+            break;
+        }
+        phases ^= 1u << st;
+        pending &= ~(1u << st);
+        const uint4 *sa = reinterpret_cast<const uint4 *>(stages + st * 2 * TILE_BYTES);
+        const uint4 *sb = reinterpret_cast<const uint4 *>(stages + st * 2 * TILE_BYTES + TILE_BYTES);
+        auto refill = [&]() {
+            __syncwarp();
+            produce(st);
+        };
+        if (n == TILE_UNITS)
+            pipe_tile<false>(sa, sb, C.u + lane, UNROLL, acc, job.s, refill);
+        else
+            pipe_tile<true>(sa, sb, C.u + lane, min(UNROLL, (n - lane + 31) / 32), acc, job.s, refill);
+        C.u += n;
+
+        if (C.u >= C.u1) {   // end of the item: warp reduction, argmax index, one partial
+            const float my_max = acc.max_a;
+            const int32_t my_best = acc.best;
+            RowPartial p = warp_reduce(acc);
+            int32_t arg = INT32_MAX;
+            if (my_max == p.max_a) {
+                const int32_t bu = my_best >> 3, bn = my_best & 7;
+                for (int j = 0; j < bn && arg == INT32_MAX; ++j) {
+                    const uint4 w4 = __ldcs(C.pa + bu + j * 32);
+                    const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+                    for (int q = 3; q >= 0; --q) {
+                        if (bf16_hi(w[q]) == my_max) arg = (bu + j * 32) * 8 + 2 * q + 1;
+                        if (bf16_lo(w[q]) == my_max) arg = (bu + j * 32) * 8 + 2 * q;
+                    }
                 }
             }
-            atomicMin(&sm.arg, arg);
+            arg = warp_min_i32(arg);
+            if (lane == 0) {
+                p.argmax = arg;
+                job.partials[C.item] = p;
+            }
+            acc.reset();
+            __syncwarp();
+            const uint32_t nx = item_ring[warp][consumed % ITEM_RING];
+            ++consumed;
+            open_item(job, C, nx);
         }
-        finish_end(sm, job.partials + item);
-        buf ^= 1;
-        item = sm.item[buf];
+        st = (st + 1 == PIPE_STAGES) ? 0 : st + 1;
     }
 }
 
@@ -197,16 +282,14 @@ __device__ __forceinline__ float load_logit<uint16_t>(const uint16_t *p, size_t 
 template <typename T>
 __global__ void __launch_bounds__(ROW_THREADS, 4) row_reduce_generic_kernel(const RowJob job)
 {
-    __shared__ ItemSmem sm;
-
-    const int tid = threadIdx.x;
-    if (tid == 0) sm.item[0] = fetch_item(job);
-    __syncthreads();
-    uint32_t item = sm.item[0];
-    int buf = 0;
+    const int lane = threadIdx.x & 31;
+    uint32_t item = 0;
+    if (lane == 0) item = fetch_item(job);
+    item = __shfl_sync(0xffffffffu, item, 0);
 
     while (item < job.total_items) {
-        if (tid == 0) sm.item[buf ^ 1] = fetch_item(job);
+        uint32_t next = 0;
+        if (lane == 0) next = fetch_item(job);   // consumed after this item
 
         const uint32_t row = item / (uint32_t)job.segments;
         const int32_t seg = (int32_t)(item % (uint32_t)job.segments);
@@ -218,19 +301,21 @@ __global__ void __launch_bounds__(ROW_THREADS, 4) row_reduce_generic_kernel(cons
         RowAcc acc;
         acc.reset();
         int32_t arg = INT32_MAX;
-        for (int32_t v = v0 + tid; v < v1; v += ROW_THREADS) {
+        for (int32_t v = v0 + lane; v < v1; v += 32) {
             const float a = load_logit<T>(pa, v), b = load_logit<T>(pb, v);
             acc.guard(a, b, job.s);
-            if (a > acc.max_a) { acc.max_a = a; arg = v; }
-            acc.add_pair(a, b, job.s, 0);
+            if (a > acc.max_a) { acc.max_a = a; arg = v; }   // strict: first occurrence within the lane
+            acc.add_pair(a, b, job.s);
             acc.flush();
         }
         const float my_max = acc.max_a;
-        const float row_max = finish_begin(acc, sm);
-        if (my_max == row_max) atomicMin(&sm.arg, arg);
-        finish_end(sm, job.partials + item);
-        buf ^= 1;
-        item = sm.item[buf];
+        RowPartial p = warp_reduce(acc);
+        arg = warp_min_i32(my_max == p.max_a ? arg : INT32_MAX);
+        if (lane == 0) {
+            p.argmax = arg;
+            job.partials[item] = p;
+        }
+        item = __shfl_sync(0xffffffffu, next, 0);
     }
 }
 
@@ -254,13 +339,6 @@ __device__ __forceinline__ double raw_logit(const void *base, int32_t dtype, siz
 {
     if (dtype == PPOW_F32) return (double)__ldg(reinterpret_cast<const float *>(base) + idx);
     return (double)__uint_as_float(((uint32_t)__ldg(reinterpret_cast<const uint16_t *>(base) + idx)) << 16);
-}
-
-__device__ __forceinline__ double warp_sum_f64(double v)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
 }
 
 constexpr int SCAN_THREADS = 128;
@@ -301,8 +379,8 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
             const double pSa = (double)p.Sa + (double)p.Sa_lo, pSb = (double)p.Sb + (double)p.Sb_lo;
             const double sa = fa * pSa;
             Sa += sa;
-            E += fa * ((double)p.E + da * pSa);
-            D += fa * ((double)p.D + (da - db) * pSa);
+            E += fa * (p.E + da * pSa);
+            D += fa * (p.D + (da - db) * pSa);
             Sb += fb * pSb;
             if (p.max_a == mx) arg = min(arg, p.argmax);
         }
@@ -397,13 +475,22 @@ static bool params_ok(const ppow_params *p)
 
 // Work items per row: one for large launches, more when there are too few rows to fill the GPU.
 // Depends only on (N, K, V) so that the workspace size is a pure function of the parameters.
+#ifndef PPOW_WORKER_WARPS
+#define PPOW_WORKER_WARPS 16      // resident warps per SM of the bulk-copy kernel
+#endif
+#ifndef PPOW_ITEMS_PER_WARP
+#define PPOW_ITEMS_PER_WARP 12
+#endif
+#ifndef PPOW_MIN_ELEMS
+#define PPOW_MIN_ELEMS 8192
+#endif
 static int segments_for(const ppow_params *p)
 {
     const int64_t rows = (int64_t)p->N * p->K;
     if (rows <= 0) return 1;
-    const int64_t want_items = 148 * 4 * 8;   // ~8 items per resident CTA on a B200
+    const int64_t want_items = (int64_t)148 * PPOW_WORKER_WARPS * PPOW_ITEMS_PER_WARP;   // on a B200
+    const int64_t elems_min = PPOW_MIN_ELEMS;   // do not cut a row finer than this many logits
     int64_t seg = (want_items + rows - 1) / rows;
-    const int64_t elems_min = 4096;            // do not cut a row finer than this many logits
     const int64_t seg_cap = p->V / elems_min > 1 ? p->V / elems_min : 1;
     if (seg > seg_cap) seg = seg_cap;
     if (seg > MAX_SEGMENTS) seg = MAX_SEGMENTS;
@@ -464,26 +551,37 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
     const bool vec_ok = params->dtype == PPOW_BF16 && (params->V % 8 == 0) &&
                         ((uintptr_t)draft_logits % 16 == 0) && ((uintptr_t)target_logits % 16 == 0) &&
                         (params->V / 8 >= segments);
+    // one warp per work item in every row kernel: a grid that fills the GPU, or fewer CTAs when there is little work
     int per_sm = 0;
     cudaError_t e;
-    if (vec_ok)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_reduce_bf16_vec_kernel, ROW_THREADS, 0);
+    int threads = ROW_THREADS;
+    size_t dyn_smem = 0;
+    if (vec_ok) {
+        threads = PIPE_WARPS * 32;
+        dyn_smem = PIPE_SMEM_BYTES;
+        e = cudaFuncSetAttribute(row_reduce_bf16_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)PIPE_SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_reduce_bf16_pipe_kernel, threads, dyn_smem);
+    }
     else if (params->dtype == PPOW_BF16)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_reduce_generic_kernel<uint16_t>, ROW_THREADS, 0);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_reduce_generic_kernel<uint16_t>, threads, 0);
     else
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_reduce_generic_kernel<float>, ROW_THREADS, 0);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_reduce_generic_kernel<float>, threads, 0);
     if (e != cudaSuccess || per_sm < 1) return PPOW_ERR_CUDA;
+    const unsigned warps_per_cta = (unsigned)threads / 32;
+    const unsigned ctas_needed = (rj.total_items + warps_per_cta - 1) / warps_per_cta;
     unsigned grid = (unsigned)(sms * per_sm);
-    if (grid > rj.total_items) grid = rj.total_items;
+    if (grid > ctas_needed) grid = ctas_needed;
 
     if (event_reduce_begin && cudaEventRecord((cudaEvent_t)event_reduce_begin, stream) != cudaSuccess)
         return PPOW_ERR_CUDA;
     if (vec_ok)
-        row_reduce_bf16_vec_kernel<<<grid, ROW_THREADS, 0, stream>>>(rj);
+        row_reduce_bf16_pipe_kernel<<<grid, threads, dyn_smem, stream>>>(rj);
     else if (params->dtype == PPOW_BF16)
-        row_reduce_generic_kernel<uint16_t><<<grid, ROW_THREADS, 0, stream>>>(rj);
+        row_reduce_generic_kernel<uint16_t><<<grid, threads, 0, stream>>>(rj);
     else
-        row_reduce_generic_kernel<float><<<grid, ROW_THREADS, 0, stream>>>(rj);
+        row_reduce_generic_kernel<float><<<grid, threads, 0, stream>>>(rj);
     if (cudaGetLastError() != cudaSuccess) return PPOW_ERR_CUDA;
     if (event_reduce_end && cudaEventRecord((cudaEvent_t)event_reduce_end, stream) != cudaSuccess)
         return PPOW_ERR_CUDA;
