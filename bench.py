@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ppow", choices=["ppow", "reference"])
     ap.add_argument("--workload", default="llama3_like", choices=[w.name for w in W.WORKLOADS])

@@ -68,15 +68,9 @@ __device__ __forceinline__ int32_t warp_min_i32(int32_t v)
 // computes on one tile, the copies of the next PIPE_STAGES - 1 tiles are in flight, across the end of
 // an item into the next one.  Loads never pause for the arithmetic, the end-of-item reduction or the
 // argmax re-read, and they hold no registers while in flight.
-#ifndef PIPE_WARPS
-#define PIPE_WARPS 8
-#endif
-#ifndef PIPE_STAGES
-#define PIPE_STAGES 3
-#endif
-#ifndef PIPE_MIN_CTAS
-#define PIPE_MIN_CTAS 2
-#endif
+constexpr int PIPE_WARPS = 8;                 // warps per CTA
+constexpr int PIPE_STAGES = 3;                // tiles per warp: one being computed on, two in flight
+constexpr int PIPE_MIN_CTAS = 2;              // 2 CTAs * 8 warps * 3 stages * 4 KB = 192 KB of shared memory per SM
 constexpr int TILE_UNITS = 32 * UNROLL;       // 16-byte units per tile per tensor
 constexpr int TILE_BYTES = TILE_UNITS * 16;   // 2 KB per tensor
 constexpr int ITEM_RING = 8;                  // > PIPE_STAGES + 1 item ids between producer and consumer
@@ -473,26 +467,21 @@ static bool params_ok(const ppow_params *p)
     return true;
 }
 
-// Work items per row: one for large launches, more when there are too few rows to fill the GPU.
-// Depends only on (N, K, V) so that the workspace size is a pure function of the parameters.
-#ifndef PPOW_WORKER_WARPS
-#define PPOW_WORKER_WARPS 16      // resident warps per SM of the bulk-copy kernel
-#endif
-#ifndef PPOW_ITEMS_PER_WARP
-#define PPOW_ITEMS_PER_WARP 12
-#endif
-#ifndef PPOW_MIN_ELEMS
-#define PPOW_MIN_ELEMS 8192
-#endif
+// Work items per row; depends only on (N, K, V) so that the workspace size is a pure function of
+// the parameters.  Measured on B200: an item should be as long as the balance allows (every item
+// ends with a warp reduction), so a row is cut only (a) to keep an item at or below about 64 tiles
+// of 1024 logits, and (b) to give each resident warp about four items when there are few rows;
+// never finer than 4 tiles.
+constexpr int64_t WORKER_WARPS = 148 * PIPE_MIN_CTAS * PIPE_WARPS;   // resident warps of the bulk-copy kernel on a B200
 static int segments_for(const ppow_params *p)
 {
     const int64_t rows = (int64_t)p->N * p->K;
     if (rows <= 0) return 1;
-    const int64_t want_items = (int64_t)148 * PPOW_WORKER_WARPS * PPOW_ITEMS_PER_WARP;   // on a B200
-    const int64_t elems_min = PPOW_MIN_ELEMS;   // do not cut a row finer than this many logits
-    int64_t seg = (want_items + rows - 1) / rows;
-    const int64_t seg_cap = p->V / elems_min > 1 ? p->V / elems_min : 1;
-    if (seg > seg_cap) seg = seg_cap;
+    const int64_t tiles = ((int64_t)p->V + 1023) / 1024;   // per row
+    int64_t seg = (4 * WORKER_WARPS + rows - 1) / rows;
+    const int64_t by_size = (tiles + 63) / 64;
+    if (seg < by_size) seg = by_size;
+    if (seg > tiles / 4) seg = tiles / 4;
     if (seg > MAX_SEGMENTS) seg = MAX_SEGMENTS;
     if (seg < 1) seg = 1;
     return (int)seg;
