@@ -30,6 +30,10 @@ import torch
 from paper_2605_14978_b200 import workloads as W
 
 METRIC = "windows/s and logit GB/s (% of B200 HBM peak) at V=128256, K=8, N=2048"
+# DRAM bytes (read + write) per window of the row-reduction kernel from the ncu capture summarised in
+# profiles/row_reduce_bf16_pipe_llama3_like.md (256-window case; traffic grows in proportion to the
+# windows processed).  Only valid for that kernel on that workload shape.
+NCU_TRAFFIC_BYTES_PER_WINDOW = {"llama3_like": 4138559.0}
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
@@ -332,7 +336,9 @@ def run_ppow(args):
         "logit_gbs": world * algo_bytes / (step_ms * 1e-3) / 1e9,
         "roofline": {"bound": "hbm", "kernel": "row_reduce", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                     "traffic": None, "algorithmic_bytes_per_launch": algo_bytes, "kernel_ms": reduce_avg_ms},
+                     "traffic": (NCU_TRAFFIC_BYTES_PER_WINDOW[w.name] * N if w.name in NCU_TRAFFIC_BYTES_PER_WINDOW else None),
+                     "traffic_source": "ncu dram__bytes_read+write on a 256-window capture, scaled by windows",
+                     "algorithmic_bytes_per_launch": algo_bytes, "kernel_ms": reduce_avg_ms},
         "e2e": e2e, "cpu_baseline": cpu_baseline, "gpu_launches": 3 * args.steps, "clocks": clocks,
         "error_flags": flags,
     }
