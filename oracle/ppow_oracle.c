@@ -26,6 +26,9 @@
  *
  * Pinned by tests/test_oracle_*.py against scipy/torch-float64 library routines, closed forms,
  * the paper's printed reward column and worked examples, brute force and invariants.
+ * The training-side quantities at the end of this file (reverse KL, expected acceptance, nabla,
+ * group-relative advantage, sliding window scores and the proportional draw of a start) are pinned by
+ * tests/test_oracle_training_pins.py.
  * Parity unpinned: Delta with a caller-supplied ref_logp (only its arithmetic is checked; producing
  * ref_logp needs a target model).
  */
@@ -277,4 +280,155 @@ int ppow_oracle_select(const double *score, int32_t N, int32_t n_keep, int32_t *
     }
     free(order);
     return 0;
+}
+
+/* =====================================================================================
+ * Training-side quantities next to the scoring pass
+ *
+ *   KL(Q_t || P_t) = sum_v Q_t(v) (log Q_t(v) - log P_t(v))      target-anchored regulariser: token-wise KL between
+ *                                                                 the draft and target distributions at each drafted
+ *                                                                 position, averaged over the window (Sec. 4.1 objective,
+ *                                                                 App. A.2)
+ *   expected acceptance = sum_v min(P_t(v), Q_t(v)) = 1 - TV     (App. B.1)
+ *   nabla = exp(d) - d - 1,  d = log P_t(yhat_t) - log Q_t(yhat_t)   alignment divergence on drafted tokens (App. E)
+ *   A_i = (R_i - mu_R) / (sigma_R + delta)                        group-relative advantage over a rollout group
+ *                                                                 (Sec. 4.1); sigma_R is the population standard
+ *                                                                 deviation of the group (reading: 1/G, not 1/(G-1))
+ *   s_j = (1/K) sum_{t=j}^{j+K-1} v_t,  j = 0..T-K                window scores over one response (Sec. 4.2; Alg. 1)
+ *   j* ~ s_j / sum_i s_i                                          Alg. 1 "Sample a training window start"; drawn by
+ *                                                                 inverse CDF from a caller-supplied uniform
+ * ===================================================================================== */
+
+typedef struct {
+    int32_t N, K, V, dtype;
+    double temperature;
+    const void *draft_logits, *target_logits;
+    const int32_t *draft_tokens, *valid_len;
+    double *kl_rev, *kl_rev_mean, *nabla, *expected_accept;
+    int32_t n_begin, n_end;
+    int status;
+} diag_slice;
+
+static void *diag_run(void *arg)
+{
+    diag_slice *s = (diag_slice *)arg;
+    const int32_t K = s->K, V = s->V;
+    double *buf = (double *)malloc(sizeof(double) * (size_t)V * 6);
+    if (!buf) { s->status = 1; return NULL; }
+    double *xa = buf, *P = buf + V, *logP = buf + 2 * (size_t)V;
+    double *xb = buf + 3 * (size_t)V, *Q = buf + 4 * (size_t)V, *logQ = buf + 5 * (size_t)V;
+    for (int32_t n = s->n_begin; n < s->n_end; ++n) {
+        int32_t L = s->valid_len ? s->valid_len[n] : K;
+        if (L < 0) L = 0;
+        if (L > K) L = K;
+        double sum_rev = 0.0;
+        for (int32_t t = 0; t < K; ++t) {
+            size_t i = (size_t)n * K + t;
+            if (t >= L) { s->kl_rev[i] = s->nabla[i] = s->expected_accept[i] = 0.0; continue; }
+            size_t row_off = i * (size_t)V;
+            (void)row_distribution(s->target_logits, s->dtype, row_off, V, s->temperature, xa, P, logP);
+            (void)row_distribution(s->draft_logits, s->dtype, row_off, V, s->temperature, xb, Q, logQ);
+            double rev = 0.0, acc = 0.0;
+            for (int32_t v = 0; v < V; ++v) {
+                if (Q[v] > 0.0) rev += Q[v] * (logQ[v] - logP[v]);
+                acc += (P[v] < Q[v]) ? P[v] : Q[v];
+            }
+            int32_t tok = s->draft_tokens[i];
+            double nab;
+            if (tok < 0 || tok >= V) nab = INFINITY;   /* not a vocabulary entry: no alignment at all */
+            else {
+                double d = logP[tok] - logQ[tok];
+                nab = expm1(d) - d;                    /* exp(d) - d - 1 without cancellation near d = 0 */
+            }
+            s->kl_rev[i] = rev;
+            s->nabla[i] = nab;
+            s->expected_accept[i] = acc;
+            sum_rev += rev;
+        }
+        s->kl_rev_mean[n] = (L > 0) ? sum_rev / (double)L : 0.0;
+    }
+    free(buf);
+    s->status = 0;
+    return NULL;
+}
+
+int ppow_oracle_diagnostics(int32_t N, int32_t K, int32_t V, int32_t dtype, double temperature,
+                            const void *draft_logits, const void *target_logits,
+                            const int32_t *draft_tokens, const int32_t *valid_len,
+                            double *kl_rev, double *kl_rev_mean, double *nabla, double *expected_accept,
+                            int32_t n_threads)
+{
+    if (N < 0 || K < 1 || V < 2 || !(temperature > 0.0)) return 2;
+    if (dtype != ORACLE_F32 && dtype != ORACLE_BF16) return 2;
+    if (N == 0) return 0;
+    if (n_threads < 1) n_threads = 1;
+    if (n_threads > N) n_threads = N;
+    pthread_t *tid = (pthread_t *)malloc(sizeof(pthread_t) * (size_t)n_threads);
+    diag_slice *sl = (diag_slice *)malloc(sizeof(diag_slice) * (size_t)n_threads);
+    if (!tid || !sl) { free(tid); free(sl); return 1; }
+    int rc = 0, started = 0;
+    for (int i = 0; i < n_threads; ++i) {
+        diag_slice d = { N, K, V, dtype, temperature, draft_logits, target_logits, draft_tokens, valid_len,
+                         kl_rev, kl_rev_mean, nabla, expected_accept,
+                         (int32_t)(((int64_t)N * i) / n_threads), (int32_t)(((int64_t)N * (i + 1)) / n_threads), 0 };
+        sl[i] = d;
+        if (n_threads == 1) diag_run(&sl[i]);
+        else if (pthread_create(&tid[i], NULL, diag_run, &sl[i]) != 0) { rc = 1; break; }
+        else ++started;
+    }
+    for (int i = 0; i < started; ++i) pthread_join(tid[i], NULL);
+    for (int i = 0; i < n_threads; ++i) if (sl[i].status) rc = 1;
+    free(tid);
+    free(sl);
+    return rc;
+}
+
+/* Group-relative advantage over contiguous groups of G windows (N must be a multiple of G). */
+int ppow_oracle_group_advantage(const double *reward, int32_t N, int32_t G, double delta, double *advantage)
+{
+    if (N < 0 || G < 1 || N % G != 0 || !(delta >= 0.0)) return 2;
+    for (int32_t g0 = 0; g0 < N; g0 += G) {
+        double mu = 0.0;
+        for (int32_t i = 0; i < G; ++i) mu += reward[g0 + i];
+        mu /= (double)G;
+        double var = 0.0;
+        for (int32_t i = 0; i < G; ++i) var += (reward[g0 + i] - mu) * (reward[g0 + i] - mu);
+        double sigma = sqrt(var / (double)G);
+        for (int32_t i = 0; i < G; ++i) advantage[g0 + i] = (reward[g0 + i] - mu) / (sigma + delta);
+    }
+    return 0;
+}
+
+/* Window scores of every start j = 0..T-K of one response; returns the number of starts (0 if T < K). */
+int32_t ppow_oracle_sliding_scores(const double *v, int32_t T, int32_t K, double *s)
+{
+    if (K < 1 || T < K) return 0;
+    for (int32_t j = 0; j + K <= T; ++j) {
+        double sum = 0.0;
+        for (int32_t t = j; t < j + K; ++t) sum += v[t];
+        s[j] = sum / (double)K;
+    }
+    return T - K + 1;
+}
+
+/* Inverse-CDF draw of a start index with probability s_j / sum s: the first j whose running sum
+ * exceeds u * total (zero-weight starts are never drawn).  All-zero weights: uniform, floor(u * n).
+ * Returns -1 when there is no start. */
+int32_t ppow_oracle_sample_start(const double *s, int32_t n, double u)
+{
+    if (n <= 0) return -1;
+    double total = 0.0;
+    for (int32_t j = 0; j < n; ++j) total += s[j];
+    if (!(total > 0.0)) {
+        int32_t j = (int32_t)(u * (double)n);
+        return j < n ? j : n - 1;
+    }
+    double run = 0.0, thresh = u * total;
+    int32_t last_positive = 0;
+    for (int32_t j = 0; j < n; ++j) {
+        run += s[j];
+        if (s[j] > 0.0) last_positive = j;
+        if (run > thresh) return j;
+    }
+    return last_positive;   /* rounding left the running sum at or below the threshold */
 }

@@ -55,6 +55,14 @@ def _load():
         lib.ppow_oracle_select.argtypes = [P, ctypes.c_int32, ctypes.c_int32, P, P]
         lib.ppow_oracle_tau_cumprod.restype = ctypes.c_int32
         lib.ppow_oracle_tau_cumprod.argtypes = [P, ctypes.c_int32]
+        lib.ppow_oracle_diagnostics.restype = ctypes.c_int
+        lib.ppow_oracle_diagnostics.argtypes = [ctypes.c_int32] * 4 + [ctypes.c_double] + [P] * 8 + [ctypes.c_int32]
+        lib.ppow_oracle_group_advantage.restype = ctypes.c_int
+        lib.ppow_oracle_group_advantage.argtypes = [P, ctypes.c_int32, ctypes.c_int32, ctypes.c_double, P]
+        lib.ppow_oracle_sliding_scores.restype = ctypes.c_int32
+        lib.ppow_oracle_sliding_scores.argtypes = [P, ctypes.c_int32, ctypes.c_int32, P]
+        lib.ppow_oracle_sample_start.restype = ctypes.c_int32
+        lib.ppow_oracle_sample_start.argtypes = [P, ctypes.c_int32, ctypes.c_double]
         _lib = lib
     return _lib
 
@@ -149,3 +157,53 @@ def tau_cumprod(flags):
     lib = _load()
     f = _np(flags, np.uint8)
     return int(lib.ppow_oracle_tau_cumprod(_ptr(f), int(f.shape[0])))
+
+
+def diagnostics(draft_logits, target_logits, draft_tokens, *, temperature=1.0, valid_len=None, n_threads=None):
+    """Per position: KL(Q||P) (``kl_rev``), expected acceptance sum_v min(P,Q) (``expected_accept``) and the
+    alignment divergence exp(d)-d-1 on the drafted token (``nabla``); per window the mean of kl_rev over the
+    valid positions (``kl_rev_mean``).  All float64."""
+    lib = _load()
+    d, dt_d = _as_numpy_logits(draft_logits)
+    t, dt_t = _as_numpy_logits(target_logits)
+    assert dt_d == dt_t and d.shape == t.shape and d.ndim == 3
+    N, K, V = d.shape
+    tok = _np(draft_tokens, np.int32)
+    vl = _np(valid_len, np.int32)
+    out = {"kl_rev": np.zeros((N, K)), "kl_rev_mean": np.zeros((N,)), "nabla": np.zeros((N, K)),
+           "expected_accept": np.zeros((N, K))}
+    rc = lib.ppow_oracle_diagnostics(N, K, V, dt_d, float(temperature), _ptr(d), _ptr(t), _ptr(tok), _ptr(vl),
+                                     _ptr(out["kl_rev"]), _ptr(out["kl_rev_mean"]), _ptr(out["nabla"]),
+                                     _ptr(out["expected_accept"]), int(n_threads or os.cpu_count() or 1))
+    if rc != 0:
+        raise RuntimeError("ppow_oracle_diagnostics failed with code %d" % rc)
+    return out
+
+
+def group_advantage(reward, group_size, delta=1e-6):
+    """(R_i - mean) / (population std + delta) within contiguous groups of ``group_size`` windows."""
+    lib = _load()
+    r = _np(reward, np.float64)
+    adv = np.zeros_like(r)
+    rc = lib.ppow_oracle_group_advantage(_ptr(r), int(r.shape[0]), int(group_size), float(delta), _ptr(adv))
+    if rc != 0:
+        raise RuntimeError("ppow_oracle_group_advantage failed with code %d" % rc)
+    return adv
+
+
+def sliding_scores(v, K):
+    """s_j = mean(v[j:j+K]) for every start j of one response (empty if it is shorter than K)."""
+    lib = _load()
+    v = _np(v, np.float64)
+    T = int(v.shape[0])
+    s = np.zeros((max(T - K + 1, 0),))
+    n = lib.ppow_oracle_sliding_scores(_ptr(v), T, int(K), _ptr(s) if s.size else None)
+    assert n == s.shape[0]
+    return s
+
+
+def sample_start(s, u):
+    """Start index drawn with probability s_j / sum(s) by inverse CDF from the uniform ``u`` (-1: no start)."""
+    lib = _load()
+    s = _np(s, np.float64)
+    return int(lib.ppow_oracle_sample_start(_ptr(s) if s.size else None, int(s.shape[0]), float(u)))
