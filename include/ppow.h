@@ -80,6 +80,14 @@ typedef struct {
     float *logp_tok;         /* [N,K] log P_t(yhat_t); -inf for an out-of-range token */
     float *logq_tok;         /* [N,K] log Q_t(yhat_t); -inf for an out-of-range token */
     int32_t *target_argmax;  /* [N,K] argmax_v of the stored target logits, lowest index on ties */
+    /* training-side quantities; asking for kl_rev or kl_rev_mean adds one fused multiply-add per logit pair */
+    float *kl_rev;           /* [N,K] KL(Q_t || P_t), nats: the target-anchored regulariser's token-wise term
+                                      (Sec. 4.1 objective; App. A.2) */
+    float *kl_rev_mean;      /* [N]   its mean over the valid positions of the window (App. A.2) */
+    float *nabla;            /* [N,K] alignment divergence exp(d) - d - 1, d = log P_t(yhat_t) - log Q_t(yhat_t)
+                                      (App. E); +inf for an out-of-range token */
+    float *lse_p;            /* [N,K] log sum_v exp(target/T), the softmax normaliser of P_t (Sec. 4.2) */
+    float *lse_q;            /* [N,K] log sum_v exp(draft/T), that of Q_t; both are inputs of ppow_expected_acceptance */
 } ppow_outputs;
 
 /* Bytes of device scratch ppow_score_windows needs for these parameters (0 on invalid params). */
@@ -151,6 +159,53 @@ ppow_status ppow_score_windows_noalloc(const ppow_params *params,
                                        const int32_t *valid_len, const float *ref_logp,
                                        const ppow_outputs *out, void *cuda_stream);
 
+/*
+ * Group-relative advantage (Sec. 4.1): for every contiguous group of `group_size` windows (one rollout
+ * group: G_roll drafts of the same prefix; the paper uses 8),
+ *     advantage[i] = (reward[i] - mu) / (sigma + delta)
+ * with mu and sigma the mean and the population standard deviation (divisor G) of the group's rewards
+ * and delta >= 0 the stabiliser.  Computed in float64, stored as float32.
+ *   reward, advantage   device, [N] float32 (may not alias)
+ * Requires N >= 0, 1 <= group_size <= 1024 and N a multiple of group_size.  No workspace.
+ */
+ppow_status ppow_group_advantage(const float *reward, int32_t N, int32_t group_size, float delta,
+                                 float *advantage, void *cuda_stream);
+
+/*
+ * Sequence form of Adaptive Divergence-Aware Windowing (Sec. 4.2; Alg. 1 "ADAW-based window selection"):
+ * for B responses stored back to back, response b owning positions [seq_offsets[b], seq_offsets[b+1]) of
+ * `crit` (the per-position criticality v_t, e.g. the crit output of ppow_score_windows), computes for every
+ * start j with a full window inside the response
+ *     scores[seq_offsets[b] + j] = (1/K) * sum_{t=j}^{j+K-1} v_t          (s_j)
+ * (0 at the last K-1 positions of a response, where no window starts), and draws one start per response
+ * with probability s_j / sum_i s_i by inverse CDF from the caller's uniform u_b in [0,1): the first j whose
+ * running sum of s exceeds u_b * sum_i s_i.  A response whose scores are all 0 draws floor(u_b * n_b)
+ * (uniform); a response shorter than K has no start (-1).  Sums run in float64 in index order.
+ *   crit          device, [seq_offsets[B]] float32, values >= 0
+ *   seq_offsets   device, [B+1] int32, non-decreasing, seq_offsets[0] = 0
+ *   scores        device, same length as crit, or NULL
+ *   uniforms      device, [B] float32, or NULL iff starts is NULL
+ *   starts        device, [B] int32 (start index relative to its response), or NULL
+ * Requires B >= 0 and 1 <= K <= 1024.  No workspace.  One thread block per response.
+ */
+ppow_status ppow_sequence_windows(const float *crit, const int32_t *seq_offsets, int32_t B, int32_t K,
+                                  float *scores, const float *uniforms, int32_t *starts, void *cuda_stream);
+
+/*
+ * Expected acceptance probability per position (App. B.1): sum_v min(P_t(v), Q_t(v)) = 1 - TV(P_t, Q_t),
+ * the probability that a token drafted from Q_t passes verification.  A second streaming pass over both
+ * logit tensors that needs the softmax normalisers of the first: lse_p, lse_q as written by
+ * ppow_score_windows (same params, same tensors).
+ *   draft_logits, target_logits, valid_len   as for ppow_score_windows
+ *   lse_p, lse_q       device, [N,K] float32
+ *   expected_accept    device, [N,K] float32; 0 at positions t >= valid_len[n]
+ * No workspace.
+ */
+ppow_status ppow_expected_acceptance(const ppow_params *params,
+                                     const void *draft_logits, const void *target_logits,
+                                     const int32_t *valid_len, const float *lse_p, const float *lse_q,
+                                     float *expected_accept, void *cuda_stream);
+
 /* Copies the error word that the last ppow_score_windows call on `workspace` left behind into
  * *flags_host (PPOW_FLAG_* bits) and synchronises `cuda_stream` to do so.  Returns
  * PPOW_ERR_DEVICE_TIMEOUT if that bit is set, PPOW_ERR_CUDA on a CUDA failure, else PPOW_OK. */
@@ -184,6 +239,8 @@ ppow_status ppow_select_windows(const float *score, int32_t N, int32_t n_keep,
  *     (may be NULL) are host pointers; pinned memory lets the copies run asynchronously;
  *   - device_scratch is device memory, 256-byte aligned, of at least
  *     ppow_host_scratch_bytes(params, 1) bytes; ppow_host_scratch_bytes(params, N) avoids chunking.
+ * Of *out_host, the outputs from accept_flag to target_argmax are served; the training-side ones
+ * after them (kl_rev, kl_rev_mean, nabla, lse_p, lse_q) are ignored by this entry point.
  * All copies and kernels are enqueued on `cuda_stream`; results are valid once it has been
  * synchronised.  The token-range error flag is not reported by this entry point (an out-of-range
  * token still shows as logp_tok = -inf and a rejected position).

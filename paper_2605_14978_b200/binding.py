@@ -24,12 +24,18 @@ PPOW_FLAG_TOKEN_RANGE, PPOW_FLAG_DEVICE_TIMEOUT = 1, 2
 EXPORTS = ("ppow_score_workspace_bytes", "ppow_score_windows", "ppow_score_windows_traced", "ppow_read_error_flags",
            "ppow_select_workspace_bytes", "ppow_select_windows", "ppow_host_scratch_bytes",
            "ppow_score_and_select_host", "ppow_noalloc_scratch_bytes", "ppow_score_windows_noalloc",
+           "ppow_group_advantage", "ppow_sequence_windows", "ppow_expected_acceptance",
            "ppow_status_string", "ppow_version")
 
 POSITION_OUTPUTS = {"accept_flag": torch.uint8, "kl": torch.float32, "conf": torch.float32, "crit": torch.float32,
                     "logp_tok": torch.float32, "logq_tok": torch.float32, "target_argmax": torch.int32}
 WINDOW_OUTPUTS = {"accepted_len": torch.int32, "reward_speedup": torch.float32, "reward_dist": torch.float32,
                   "reward": torch.float32, "delta": torch.float32, "score": torch.float32}
+# training-side outputs of the scoring pass, written only when asked for
+TRAIN_POSITION_OUTPUTS = {"kl_rev": torch.float32, "nabla": torch.float32, "lse_p": torch.float32,
+                          "lse_q": torch.float32}
+TRAIN_WINDOW_OUTPUTS = {"kl_rev_mean": torch.float32}
+_ALL_OUTPUTS = {**POSITION_OUTPUTS, **WINDOW_OUTPUTS, **TRAIN_POSITION_OUTPUTS, **TRAIN_WINDOW_OUTPUTS}
 
 
 class ppow_params(ctypes.Structure):
@@ -43,7 +49,8 @@ class ppow_outputs(ctypes.Structure):
     # field order is the order of the C struct
     _fields_ = [(n, ctypes.c_void_p) for n in
                 ("accept_flag", "accepted_len", "reward_speedup", "reward_dist", "reward", "delta", "score",
-                 "kl", "conf", "crit", "logp_tok", "logq_tok", "target_argmax")]
+                 "kl", "conf", "crit", "logp_tok", "logq_tok", "target_argmax",
+                 "kl_rev", "kl_rev_mean", "nabla", "lse_p", "lse_q")]
 
 
 class PpowError(RuntimeError):
@@ -88,6 +95,12 @@ def load_library():
     lib.ppow_score_windows_noalloc.restype = ctypes.c_int
     lib.ppow_score_windows_noalloc.argtypes = [ctypes.POINTER(ppow_params), vp, vp, vp, vp, vp, vp,
                                                ctypes.POINTER(ppow_outputs), vp]
+    lib.ppow_group_advantage.restype = ctypes.c_int
+    lib.ppow_group_advantage.argtypes = [vp, i32, i32, ctypes.c_float, vp, vp]
+    lib.ppow_sequence_windows.restype = ctypes.c_int
+    lib.ppow_sequence_windows.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
+    lib.ppow_expected_acceptance.restype = ctypes.c_int
+    lib.ppow_expected_acceptance.argtypes = [ctypes.POINTER(ppow_params), vp, vp, vp, vp, vp, vp, vp]
     lib.ppow_status_string.restype = ctypes.c_char_p
     lib.ppow_status_string.argtypes = [ctypes.c_int]
     lib.ppow_version.restype = ctypes.c_int
@@ -141,6 +154,12 @@ def alloc_outputs(N: int, K: int, device) -> dict:
     return out
 
 
+def alloc_train_outputs(N: int, K: int, device) -> dict:
+    out = {k: torch.empty((N, K), dtype=dt, device=device) for k, dt in TRAIN_POSITION_OUTPUTS.items()}
+    out.update({k: torch.empty((N,), dtype=dt, device=device) for k, dt in TRAIN_WINDOW_OUTPUTS.items()})
+    return out
+
+
 def alloc_workspace(nbytes: int, device) -> torch.Tensor:
     # torch's caching allocator returns 512-byte aligned blocks
     return torch.empty((max(int(nbytes), 256),), dtype=torch.uint8, device=device)
@@ -172,7 +191,7 @@ def ppow_score_windows_traced(params: ppow_params, draft_logits, target_logits, 
     o = ppow_outputs()
     for name, _ in ppow_outputs._fields_:
         t = outputs.get(name)
-        want = POSITION_OUTPUTS.get(name) or WINDOW_OUTPUTS.get(name)
+        want = _ALL_OUTPUTS[name]
         p = _dev_ptr(t, want, name)
         setattr(o, name, p.value if p is not None else None)
     traced = event_reduce_begin is not None or event_reduce_end is not None
@@ -223,7 +242,7 @@ def ppow_score_windows_noalloc(params: ppow_params, draft_logits, target_logits,
     lt = torch.float32 if params.dtype == PPOW_F32 else torch.bfloat16
     o = ppow_outputs()
     for name, _ in ppow_outputs._fields_:
-        want = POSITION_OUTPUTS.get(name) or WINDOW_OUTPUTS.get(name)
+        want = _ALL_OUTPUTS[name]
         p = _dev_ptr(outputs.get(name), want, name)
         setattr(o, name, p.value if p is not None else None)
     st = lib.ppow_score_windows_noalloc(
@@ -234,6 +253,39 @@ def ppow_score_windows_noalloc(params: ppow_params, draft_logits, target_logits,
         ctypes.byref(o), _stream_ptr(stream))
     if st != PPOW_OK:
         raise PpowError(st, "ppow_score_windows_noalloc")
+
+
+def ppow_group_advantage(reward, group_size: int, delta: float, advantage, stream=None) -> None:
+    lib = load_library()
+    N = int(reward.numel()) if reward is not None else 0
+    st = lib.ppow_group_advantage(_dev_ptr(reward, torch.float32, "reward"), N, int(group_size), float(delta),
+                                  _dev_ptr(advantage, torch.float32, "advantage"), _stream_ptr(stream))
+    if st != PPOW_OK:
+        raise PpowError(st, "ppow_group_advantage")
+
+
+def ppow_sequence_windows(crit, seq_offsets, K: int, scores, uniforms, starts, stream=None) -> None:
+    lib = load_library()
+    B = int(seq_offsets.numel()) - 1 if seq_offsets is not None else 0
+    st = lib.ppow_sequence_windows(_dev_ptr(crit, torch.float32, "crit"), _dev_ptr(seq_offsets, torch.int32, "seq_offsets"),
+                                   B, int(K), _dev_ptr(scores, torch.float32, "scores"),
+                                   _dev_ptr(uniforms, torch.float32, "uniforms"), _dev_ptr(starts, torch.int32, "starts"),
+                                   _stream_ptr(stream))
+    if st != PPOW_OK:
+        raise PpowError(st, "ppow_sequence_windows")
+
+
+def ppow_expected_acceptance(params: ppow_params, draft_logits, target_logits, valid_len, lse_p, lse_q,
+                             expected_accept, stream=None) -> None:
+    lib = load_library()
+    lt = torch.float32 if params.dtype == PPOW_F32 else torch.bfloat16
+    st = lib.ppow_expected_acceptance(
+        ctypes.byref(params), _dev_ptr(draft_logits, lt, "draft_logits"), _dev_ptr(target_logits, lt, "target_logits"),
+        _dev_ptr(valid_len, torch.int32, "valid_len"), _dev_ptr(lse_p, torch.float32, "lse_p"),
+        _dev_ptr(lse_q, torch.float32, "lse_q"), _dev_ptr(expected_accept, torch.float32, "expected_accept"),
+        _stream_ptr(stream))
+    if st != PPOW_OK:
+        raise PpowError(st, "ppow_expected_acceptance")
 
 
 def _host_ptr(t: Optional[torch.Tensor], dtype=None, name="tensor"):
@@ -258,7 +310,7 @@ def ppow_score_and_select_host(params: ppow_params, draft_logits, target_logits,
     lt = torch.float32 if params.dtype == PPOW_F32 else torch.bfloat16
     o = ppow_outputs()
     for name, _ in ppow_outputs._fields_:
-        want = POSITION_OUTPUTS.get(name) or WINDOW_OUTPUTS.get(name)
+        want = _ALL_OUTPUTS[name]
         p = _host_ptr(outputs_host.get(name), want, name)
         setattr(o, name, p.value if p is not None else None)
     st = lib.ppow_score_and_select_host(
@@ -276,14 +328,17 @@ def ppow_score_and_select_host(params: ppow_params, draft_logits, target_logits,
 
 
 def score_windows(draft_logits, target_logits, draft_tokens, *, mode, c, temperature=1.0, eta=1.0, eps=0.5,
-                  uniforms=None, valid_len=None, ref_logp=None, stream=None) -> dict:
-    """Allocate outputs and workspace, run ppow_score_windows, return the dict of output tensors."""
+                  uniforms=None, valid_len=None, ref_logp=None, stream=None, train_outputs=False) -> dict:
+    """Allocate outputs and workspace, run ppow_score_windows, return the dict of output tensors
+    (with ``train_outputs`` also kl_rev, kl_rev_mean, nabla, lse_p, lse_q)."""
     N, K, V = draft_logits.shape
     dt = PPOW_F32 if draft_logits.dtype == torch.float32 else PPOW_BF16
     params = make_params(N, K, V, dt, mode, c, temperature, eta, eps)
     dev = draft_logits.device
     with torch.cuda.device(dev):
         out = alloc_outputs(N, K, dev)
+        if train_outputs:
+            out.update(alloc_train_outputs(N, K, dev))
         ws = alloc_workspace(ppow_score_workspace_bytes(params), dev)
         ppow_score_windows(params, draft_logits, target_logits, draft_tokens, uniforms, valid_len, ref_logp, out,
                            ws, stream)

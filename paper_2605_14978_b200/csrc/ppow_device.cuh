@@ -10,6 +10,8 @@
 // Each thread accumulates
 //   Sa = sum 2^x_a     Sb = sum 2^x_b     E = sum 2^x_a * x_a     D = sum 2^x_a * (x_a - x_b)
 // from which (Sec. 4.2)  H(P)/ln2 = log2 Sa - E/Sa  and  KL(P||Q)/ln2 = D/Sa - log2 Sa + log2 Sb.
+// When the reverse divergence of the training objective is wanted (Sec. 4.1, App. A.2) one more sum,
+//   B = sum 2^x_b * (x_a - x_b),   gives   KL(Q||P)/ln2 = -B/Sb - log2 Sb + log2 Sa.
 // Accumulating D from the per-element difference (not E - F) avoids cancelling two O(10) terms
 // to reach a KL of O(0.01).
 #pragma once
@@ -28,10 +30,11 @@ struct __align__(16) RowPartial {
     float Sa, Sb;         // sums relative to those references (leading parts)
     float Sa_lo, Sb_lo;   // their compensation terms: the sums are Sa + Sa_lo, Sb + Sb_lo
     double E, D;          // weighted sums relative to the same references
+    double B;             // sum 2^x_b (x_a - x_b), for KL(Q||P); 0 unless the call asks for it
     float max_a;          // largest stored target logit seen
     int32_t argmax;       // its lowest vocabulary index
 };
-static_assert(sizeof(RowPartial) == 48, "RowPartial layout");
+static_assert(sizeof(RowPartial) == 64, "RowPartial layout");
 
 __device__ __forceinline__ float ex2_approx(float x)
 {
@@ -61,18 +64,20 @@ __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w 
 // The tile-local accumulators are float2: lane .x takes the even vocabulary entries of a packed bf16
 // word, lane .y the odd ones, so that the arithmetic runs on sm_100's packed f32x2 instructions
 // (__ffma2_rn / __fadd2_rn: one issue slot for two IEEE fma/add operations).
+// REV: also accumulate B for KL(Q||P) (one more packed fma per word; members unused otherwise).
+template <bool REV>
 struct RowAcc {
     float rho_a, rho_b;
-    float2 Sa, Sb, E, D;
-    float Sa_hi, Sa_lo, Sb_hi, Sb_lo, E_hi, E_lo, D_hi, D_lo;
+    float2 Sa, Sb, E, D, B;
+    float Sa_hi, Sa_lo, Sb_hi, Sb_lo, E_hi, E_lo, D_hi, D_lo, B_hi, B_lo;
     float max_a;
     int32_t best;       // where max_a was first seen (meaning defined by the caller)
 
     __device__ __forceinline__ void reset()
     {
         rho_a = rho_b = RHO_INIT;
-        Sa = Sb = E = D = make_float2(0.0f, 0.0f);
-        Sa_hi = Sa_lo = Sb_hi = Sb_lo = E_hi = E_lo = D_hi = D_lo = 0.0f;
+        Sa = Sb = E = D = B = make_float2(0.0f, 0.0f);
+        Sa_hi = Sa_lo = Sb_hi = Sb_lo = E_hi = E_lo = D_hi = D_lo = B_hi = B_lo = 0.0f;
         max_a = -INFINITY;
         best = 0;
     }
@@ -93,11 +98,12 @@ struct RowAcc {
         two_sum(Sb_hi, Sb_lo, Sb.x + Sb.y);
         two_sum(E_hi, E_lo, E.x + E.y);
         two_sum(D_hi, D_lo, D.x + D.y);
-        Sa = Sb = E = D = make_float2(0.0f, 0.0f);
+        if (REV) two_sum(B_hi, B_lo, B.x + B.y);
+        Sa = Sb = E = D = B = make_float2(0.0f, 0.0f);
     }
 
     // Move both references (log2 units).  Only between tiles (after flush()).  With x' = x - d,
-    //   Sa' = fa*Sa,  E' = fa*(E + da*Sa),  D' = fa*(D + (da - db)*Sa),  Sb' = fb*Sb
+    //   Sa' = fa*Sa,  E' = fa*(E + da*Sa),  D' = fa*(D + (da - db)*Sa),  Sb' = fb*Sb,  B' = fb*(B + (da - db)*Sb)
     // where da = rho_a - new_rho_a <= 0 and fa = 2^da (same for b).  Applying (da - db) in one step
     // keeps D exactly 0 when draft and target are the same data.
     __device__ __forceinline__ void rebase(float new_rho_a, float new_rho_b)
@@ -109,6 +115,10 @@ struct RowAcc {
         E_hi = fa * fmaf(da, S, E_hi + E_lo);
         D_hi = fa * fmaf(da - db, S, D_hi + D_lo);
         E_lo = D_lo = 0.0f;
+        if (REV) {
+            B_hi = fb * fmaf(da - db, Sb_hi + Sb_lo, B_hi + B_lo);
+            B_lo = 0.0f;
+        }
         Sa_hi *= fa;
         Sa_lo *= fa;
         Sb_hi *= fb;
@@ -128,6 +138,7 @@ struct RowAcc {
         Sb.x += eb;
         E.x = fmaf(ea, xa, E.x);
         D.x = fmaf(ea, xa - xb, D.x);
+        if (REV) B.x = fmaf(eb, xa - xb, B.x);
     }
 
     // Two packed bf16 pairs: the same operations as two add_pair calls, two per instruction.
@@ -143,6 +154,7 @@ struct RowAcc {
         E = __ffma2_rn(ea, xa, E);
         const float2 dx = __ffma2_rn(xb, make_float2(-1.0f, -1.0f), xa);   // xa - xb, one rounding
         D = __ffma2_rn(ea, dx, D);
+        if (REV) B = __ffma2_rn(eb, dx, B);
     }
 
     // Raise the references if this tile's maxima (raw logit units) call for it.
@@ -190,7 +202,8 @@ __device__ __forceinline__ double warp_sum_f64(double v)
 }
 
 // Reduce a warp's accumulators to one partial (valid in every lane); argmax is left unset.
-__device__ __forceinline__ RowPartial warp_reduce(RowAcc acc)
+template <bool REV>
+__device__ __forceinline__ RowPartial warp_reduce(RowAcc<REV> acc)
 {
     const float Ra = warp_max(acc.rho_a);
     const float Rb = warp_max(acc.rho_b);
@@ -204,6 +217,7 @@ __device__ __forceinline__ RowPartial warp_reduce(RowAcc acc)
     p.Sb = acc.Sb_hi; p.Sb_lo = acc.Sb_lo;
     p.E = warp_sum_f64((double)acc.E_hi + (double)acc.E_lo);
     p.D = warp_sum_f64((double)acc.D_hi + (double)acc.D_lo);
+    p.B = REV ? warp_sum_f64((double)acc.B_hi + (double)acc.B_lo) : 0.0;
     p.max_a = warp_max(acc.max_a);
     p.argmax = INT32_MAX;
     return p;

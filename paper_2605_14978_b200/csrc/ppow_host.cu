@@ -122,7 +122,7 @@ extern "C" ppow_status ppow_score_and_select_host(const ppow_params *params,
 
         ppow_params q = *params;
         q.N = nw;
-        ppow_outputs o;
+        ppow_outputs o = {};   // outputs this entry point does not stage (kl_rev, nabla, ...) stay NULL
         o.accept_flag = out_host->accept_flag ? (uint8_t *)(cb + L.pos_u8) : nullptr;
         o.kl = out_host->kl ? (float *)(cb + L.pos_f32[0]) : nullptr;
         o.conf = out_host->conf ? (float *)(cb + L.pos_f32[1]) : nullptr;

@@ -100,8 +100,8 @@ __device__ __forceinline__ void open_item(const RowJob &job, ItemCursor &c, uint
 
 // One tile out of shared memory.  `nu` = units of this lane that exist (UNROLL unless MASKED);
 // refill() is called once every value of the stage sits in registers.
-template <bool MASKED, typename Refill>
-__device__ __forceinline__ void pipe_tile(const uint4 *sa, const uint4 *sb, int32_t u, int nu, RowAcc &acc,
+template <bool MASKED, bool REV, typename Refill>
+__device__ __forceinline__ void pipe_tile(const uint4 *sa, const uint4 *sb, int32_t u, int nu, RowAcc<REV> &acc,
                                           float s, Refill refill)
 {
     const int lane = threadIdx.x & 31;
@@ -141,6 +141,7 @@ __device__ __forceinline__ void pipe_tile(const uint4 *sa, const uint4 *sb, int3
     acc.flush();
 }
 
+template <bool REV>
 __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_bf16_pipe_kernel(const RowJob job)
 {
     extern __shared__ __align__(128) unsigned char pipe_smem[];
@@ -201,7 +202,7 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_bf1
 
     uint32_t phases = 0;
     int st = 0;
-    RowAcc acc;
+    RowAcc<REV> acc;
     acc.reset();
     while (C.item < job.total_items) {
         const int32_t n = min(TILE_UNITS, C.u1 - C.u);
@@ -224,9 +225,9 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_bf1
             produce(st);
         };
         if (n == TILE_UNITS)
-            pipe_tile<false>(sa, sb, C.u + lane, UNROLL, acc, job.s, refill);
+            pipe_tile<false, REV>(sa, sb, C.u + lane, UNROLL, acc, job.s, refill);
         else
-            pipe_tile<true>(sa, sb, C.u + lane, min(UNROLL, (n - lane + 31) / 32), acc, job.s, refill);
+            pipe_tile<true, REV>(sa, sb, C.u + lane, min(UNROLL, (n - lane + 31) / 32), acc, job.s, refill);
         C.u += n;
 
         if (C.u >= C.u1) {   // end of the item: warp reduction, argmax index, one partial
@@ -273,7 +274,7 @@ __device__ __forceinline__ float load_logit<uint16_t>(const uint16_t *p, size_t 
     return __uint_as_float(((uint32_t)__ldcs(p + i)) << 16);
 }
 
-template <typename T>
+template <typename T, bool REV>
 __global__ void __launch_bounds__(ROW_THREADS, 4) row_reduce_generic_kernel(const RowJob job)
 {
     const int lane = threadIdx.x & 31;
@@ -292,7 +293,7 @@ __global__ void __launch_bounds__(ROW_THREADS, 4) row_reduce_generic_kernel(cons
         const T *pa = reinterpret_cast<const T *>(job.target) + (size_t)row * job.V;
         const T *pb = reinterpret_cast<const T *>(job.draft) + (size_t)row * job.V;
 
-        RowAcc acc;
+        RowAcc<REV> acc;
         acc.reset();
         int32_t arg = INT32_MAX;
         for (int32_t v = v0 + lane; v < v1; v += 32) {
@@ -348,8 +349,8 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
     const bool active = lane < L;
     const double LN2 = 0.69314718055994530942;
 
-    double crit = 0.0, gap = 0.0, lp = 0.0;
-    float o_kl = 0.f, o_conf = 0.f, o_crit = 0.f, o_lp = 0.f, o_lq = 0.f;
+    double crit = 0.0, gap = 0.0, lp = 0.0, kl_rev = 0.0;
+    float o_kl = 0.f, o_conf = 0.f, o_crit = 0.f, o_lp = 0.f, o_lq = 0.f, o_nabla = 0.f, o_lse_p = 0.f, o_lse_q = 0.f;
     int32_t o_arg = 0;
     int flag = 0;
 
@@ -364,7 +365,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
             Rb = fmax(Rb, (double)pp[i].rho_b);
             mx = fmaxf(mx, pp[i].max_a);
         }
-        double Sa = 0.0, Sb = 0.0, E = 0.0, D = 0.0;
+        double Sa = 0.0, Sb = 0.0, E = 0.0, D = 0.0, Bv = 0.0;
         int32_t arg = INT32_MAX;
         for (int i = 0; i < job.segments; ++i) {
             const RowPartial p = pp[i];
@@ -376,12 +377,16 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
             E += fa * (p.E + da * pSa);
             D += fa * (p.D + (da - db) * pSa);
             Sb += fb * pSb;
+            Bv += fb * (p.B + (da - db) * pSb);
             if (p.max_a == mx) arg = min(arg, p.argmax);
         }
         const double s = (double)job.s;
         const double l2Sa = log2(Sa), l2Sb = log2(Sb);
         const double H = (l2Sa - E / Sa) * LN2;                 // entropy of P, nats
         const double KL = (D / Sa - l2Sa + l2Sb) * LN2;         // KL(P || Q), nats
+        kl_rev = (-Bv / Sb - l2Sb + l2Sa) * LN2;              // KL(Q || P), nats (meaningful only if B was accumulated)
+        o_lse_p = (float)((Ra + l2Sa) * LN2);
+        o_lse_q = (float)((Rb + l2Sb) * LN2);
         double C = 1.0 - H / log((double)job.V);
         C = fmin(1.0, fmax(0.0, C));
         crit = C * KL;
@@ -394,12 +399,14 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
             lp = -INFINITY;
             lq = -INFINITY;
             flag = 0;
+            o_nabla = INFINITY;
         } else {
             const double a_tok = raw_logit(job.target, job.dtype, row * job.V + tok);
             const double b_tok = raw_logit(job.draft, job.dtype, row * job.V + tok);
             lp2 = fma(a_tok, s, -Ra) - l2Sa;
             lp = lp2 * LN2;
             lq = (fma(b_tok, s, -Rb) - l2Sb) * LN2;
+            o_nabla = (float)(expm1(lp - lq) - (lp - lq));   // exp(d) - d - 1 without cancellation near d = 0
             if (job.mode == PPOW_GREEDY) {
                 flag = (tok == arg);
             } else {
@@ -421,6 +428,10 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
         if (job.out.logp_tok) job.out.logp_tok[row] = o_lp;
         if (job.out.logq_tok) job.out.logq_tok[row] = o_lq;
         if (job.out.target_argmax) job.out.target_argmax[row] = o_arg;
+        if (job.out.kl_rev) job.out.kl_rev[row] = (float)kl_rev;
+        if (job.out.nabla) job.out.nabla[row] = o_nabla;
+        if (job.out.lse_p) job.out.lse_p[row] = o_lse_p;
+        if (job.out.lse_q) job.out.lse_q[row] = o_lse_q;
     }
 
     // accepted length = number of leading accepted positions (App. C.1)
@@ -432,9 +443,10 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
     const double sum_crit = warp_sum_f64(crit);
     const double sum_gap = warp_sum_f64(gap);
     const double sum_lp = warp_sum_f64(lp);
+    const double sum_rev = warp_sum_f64(kl_rev);
 
     if (lane == 0) {
-        float r_speed = 0.f, r_dist = 0.f, delta = 0.f, score = 0.f;
+        float r_speed = 0.f, r_dist = 0.f, delta = 0.f, score = 0.f, rev_mean = 0.f;
         if (L > 0) {
             const double rs = (double)k / ((double)k * (double)job.c + 1.0);
             const double dl = job.ref_logp ? ((double)__ldg(job.ref_logp + n) - sum_lp) : sum_gap;
@@ -442,6 +454,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
             delta = (float)dl;
             r_dist = (k == 0 && dl < (double)job.eps) ? job.eta : 0.f;
             score = (float)(sum_crit / (double)L);
+            rev_mean = (float)(sum_rev / (double)L);
         }
         job.out.accepted_len[n] = k;
         if (job.out.reward_speedup) job.out.reward_speedup[n] = r_speed;
@@ -449,6 +462,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
         if (job.out.reward) job.out.reward[n] = r_speed + r_dist;
         if (job.out.delta) job.out.delta[n] = delta;
         if (job.out.score) job.out.score[n] = score;
+        if (job.out.kl_rev_mean) job.out.kl_rev_mean[n] = rev_mean;
     }
 }
 
@@ -540,24 +554,28 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
     const bool vec_ok = params->dtype == PPOW_BF16 && (params->V % 8 == 0) &&
                         ((uintptr_t)draft_logits % 16 == 0) && ((uintptr_t)target_logits % 16 == 0) &&
                         (params->V / 8 >= segments);
-    // one warp per work item in every row kernel: a grid that fills the GPU, or fewer CTAs when there is little work
-    int per_sm = 0;
-    cudaError_t e;
+    // one warp per work item in every row kernel: a grid that fills the GPU, or fewer CTAs when there is little work.
+    // The kernels that also accumulate the sum for KL(Q||P) run only when that output is asked for.
+    const bool rev = out->kl_rev != nullptr || out->kl_rev_mean != nullptr;
+    const void *kernel;
     int threads = ROW_THREADS;
     size_t dyn_smem = 0;
     if (vec_ok) {
+        kernel = rev ? (const void *)row_reduce_bf16_pipe_kernel<true> : (const void *)row_reduce_bf16_pipe_kernel<false>;
         threads = PIPE_WARPS * 32;
         dyn_smem = PIPE_SMEM_BYTES;
-        e = cudaFuncSetAttribute(row_reduce_bf16_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)PIPE_SMEM_BYTES);
-        if (e == cudaSuccess)
-            e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_reduce_bf16_pipe_kernel, threads, dyn_smem);
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PIPE_SMEM_BYTES) != cudaSuccess)
+            return PPOW_ERR_CUDA;
+    } else if (params->dtype == PPOW_BF16) {
+        kernel = rev ? (const void *)row_reduce_generic_kernel<uint16_t, true>
+                     : (const void *)row_reduce_generic_kernel<uint16_t, false>;
+    } else {
+        kernel = rev ? (const void *)row_reduce_generic_kernel<float, true>
+                     : (const void *)row_reduce_generic_kernel<float, false>;
     }
-    else if (params->dtype == PPOW_BF16)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_reduce_generic_kernel<uint16_t>, threads, 0);
-    else
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_reduce_generic_kernel<float>, threads, 0);
-    if (e != cudaSuccess || per_sm < 1) return PPOW_ERR_CUDA;
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, dyn_smem) != cudaSuccess || per_sm < 1)
+        return PPOW_ERR_CUDA;
     const unsigned warps_per_cta = (unsigned)threads / 32;
     const unsigned ctas_needed = (rj.total_items + warps_per_cta - 1) / warps_per_cta;
     unsigned grid = (unsigned)(sms * per_sm);
@@ -565,12 +583,9 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
 
     if (event_reduce_begin && cudaEventRecord((cudaEvent_t)event_reduce_begin, stream) != cudaSuccess)
         return PPOW_ERR_CUDA;
-    if (vec_ok)
-        row_reduce_bf16_pipe_kernel<<<grid, threads, dyn_smem, stream>>>(rj);
-    else if (params->dtype == PPOW_BF16)
-        row_reduce_generic_kernel<uint16_t><<<grid, threads, 0, stream>>>(rj);
-    else
-        row_reduce_generic_kernel<float><<<grid, threads, 0, stream>>>(rj);
+    void *kargs[] = {(void *)&rj};
+    if (cudaLaunchKernel(kernel, dim3(grid), dim3((unsigned)threads), kargs, dyn_smem, stream) != cudaSuccess)
+        return PPOW_ERR_CUDA;
     if (cudaGetLastError() != cudaSuccess) return PPOW_ERR_CUDA;
     if (event_reduce_end && cudaEventRecord((cudaEvent_t)event_reduce_end, stream) != cudaSuccess)
         return PPOW_ERR_CUDA;
