@@ -47,6 +47,10 @@ def parse_args():
     ap.add_argument("--workload", default="llama3_like", choices=[w.name for w in W.WORKLOADS])
     ap.add_argument("--mode", default=None, choices=[None, "greedy", "stochastic"])
     ap.add_argument("--windows", type=int, default=None, help="override N (small cases for profiler captures)")
+    ap.add_argument("--train", action="store_true",
+                    help="the step also produces the training-side quantities: KL(Q||P), nabla and the softmax "
+                         "normalisers from the scoring pass, the group-relative advantage (groups of 8), and the "
+                         "expected-acceptance pass (a second read of both logit tensors)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
     return ap.parse_args()
@@ -235,14 +239,31 @@ def run_ppow(args):
 
     params = B.make_params(N, K, V, B.PPOW_F32 if w.dtype == "f32" else B.PPOW_BF16, bmode, w.c, w.temperature)
     out = B.alloc_outputs(N, K, dev)
+    if args.train:
+        out.update(B.alloc_train_outputs(N, K, dev))
+        advantage = torch.empty((N,), dtype=torch.float32, device=dev)
+        exp_accept = torch.empty((N, K), dtype=torch.float32, device=dev)
+        group = 8 if N % 8 == 0 else 1
     ws = B.alloc_workspace(B.ppow_score_workspace_bytes(params), dev)
     selected = torch.empty((n_keep,), dtype=torch.int32, device=dev)
     sel_ws = B.alloc_workspace(B.ppow_select_workspace_bytes(n_total), dev)
     stream = torch.cuda.current_stream()
 
+    acc_events = []
+
     def step(ev0=None, ev1=None):
         B.ppow_score_windows_traced(params, x["draft_logits"], x["target_logits"], x["draft_tokens"], x["uniforms"],
                                     x["valid_len"], None, out, ws, stream, ev0, ev1)
+        if args.train:
+            B.ppow_group_advantage(out["reward"], group, 1e-6, advantage, stream)
+            ea, eb = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) if ev0 is not None else (None, None)
+            if ea is not None:
+                ea.record(stream)
+            B.ppow_expected_acceptance(params, x["draft_logits"], x["target_logits"], x["valid_len"], out["lse_p"],
+                                       out["lse_q"], exp_accept, stream)
+            if ea is not None:
+                eb.record(stream)
+                acc_events.append((ea, eb))
         scores = S.gather_scores(out["score"], n_total) if world > 1 else out["score"]   # the one exchange step
         B.ppow_select_windows(scores, n_keep, selected, None, sel_ws, stream)
 
@@ -339,7 +360,12 @@ def run_ppow(args):
                      "traffic": (NCU_TRAFFIC_BYTES_PER_WINDOW[w.name] * N if w.name in NCU_TRAFFIC_BYTES_PER_WINDOW else None),
                      "traffic_source": "ncu dram__bytes_read+write on a 256-window capture, scaled by windows",
                      "algorithmic_bytes_per_launch": algo_bytes, "kernel_ms": reduce_avg_ms},
-        "e2e": e2e, "cpu_baseline": cpu_baseline, "gpu_launches": 3 * args.steps, "clocks": clocks,
+        "training": ({"kl_rev_in_scoring_pass": True, "group_size": group,
+                      "expected_acceptance_ms": sum(a.elapsed_time(b) for a, b in acc_events) / len(acc_events),
+                      "expected_acceptance_gbs": algo_bytes / (sum(a.elapsed_time(b) for a, b in acc_events)
+                                                               / len(acc_events) * 1e-3) / 1e9}
+                     if args.train else None),
+        "e2e": e2e, "cpu_baseline": cpu_baseline, "gpu_launches": (5 if args.train else 3) * args.steps, "clocks": clocks,
         "error_flags": flags,
     }
     print(json.dumps(line))
