@@ -193,6 +193,22 @@ def test_extreme_rows_exercise_reference_rebasing():
     _both_modes(x)
 
 
+@pytest.mark.parametrize("top", [12.0, 15.5, 16.5, 17.5])
+def test_one_confident_token_over_a_flat_tail(top):
+    """The hardest case for single-precision sums: one term decides the sum and 128255 equal terms, each
+    near half an ulp of it, follow.  Every add after the big term rounds the same way, so the error grows
+    with the number of adds between two compensated folds; this pins that interval."""
+    N, K, V = 4, 8, 128256
+    g = torch.Generator(device=DEV).manual_seed(int(top * 10))
+    pos = torch.randint(0, V // 8, (N, K), generator=g, device=DEV) * 8      # first logit of a 16-byte unit
+    t = torch.zeros((N, K, V), device=DEV).scatter_(2, pos[..., None], top).to(torch.bfloat16)
+    d = torch.zeros((N, K, V), device=DEV).scatter_(2, pos[..., None], top - 1.0).to(torch.bfloat16)
+    x = {"target_logits": t, "draft_logits": d, "draft_tokens": pos.to(torch.int32),
+         "uniforms": torch.rand((N, K), generator=g, device=DEV), "valid_len": None}
+    gpu, ref = _both_modes(x, c=0.04)
+    assert bool((gpu["target_argmax"] == pos).all())
+
+
 def test_reference_window_logprob_variant_of_delta():
     x = _random_inputs(9, 5, 2048, torch.bfloat16, seed=11, sigma=0.2)
     ref_logp = -torch.rand(9, device=DEV) * 3.0
