@@ -140,7 +140,7 @@ ppow_status ppow_score_windows_traced(const ppow_params *params,
  * no counterpart.)  For callers that cannot obtain device scratch memory: code that runs beside a
  * framework which already owns all device memory and whose allocator it cannot reach, or code
  * that must not allocate after start-up.  The scratch is a fixed array of
- * ppow_noalloc_scratch_bytes() (2 MiB) of device global memory inside the library image; every GPU
+ * ppow_noalloc_scratch_bytes() (4 MiB) of device global memory inside the library image; every GPU
  * that loads the library holds it until the process exits.  Inputs, outputs, stream and results
  * are exactly those of ppow_score_windows.  No memory is allocated or freed by this call.
  *   - Returns PPOW_ERR_UNSUPPORTED, launching nothing, when

@@ -235,7 +235,7 @@ def ppow_noalloc_scratch_bytes() -> int:
 
 def ppow_score_windows_noalloc(params: ppow_params, draft_logits, target_logits, draft_tokens, uniforms, valid_len,
                                ref_logp, outputs: dict, stream=None) -> None:
-    """ppow_score_windows for callers that cannot hand over a workspace: the library's built-in 2 MiB
+    """ppow_score_windows for callers that cannot hand over a workspace: the library's built-in 4 MiB
     scratch array is used instead.  The binding itself allocates nothing here; ``outputs`` must hold
     preallocated CUDA tensors.  Calls on one device must not overlap (they share the array)."""
     lib = load_library()

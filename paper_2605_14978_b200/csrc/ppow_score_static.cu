@@ -22,7 +22,7 @@
 
 #include <mutex>
 
-#define PPOW_NOALLOC_SCRATCH_BYTES (2u * 1024u * 1024u)
+#define PPOW_NOALLOC_SCRATCH_BYTES (4u * 1024u * 1024u)
 #define PPOW_NOALLOC_MAX_DEVICES 64
 
 // In host code this name is only a handle for the runtime's symbol lookup, not a device address.

@@ -2,7 +2,7 @@
 
 Some users of the library sit beside a framework that has already claimed the device's memory and
 whose allocator they cannot reach (a plain-C plugin, a scheduler thread), or must not allocate once
-a run has started.  They call this entry point, which uses a fixed 2 MiB array inside the library
+a run has started.  They call this entry point, which uses a fixed 4 MiB array inside the library
 instead of a caller-provided workspace.  The test calls it through the C ABI twice in a row (the
 array is shared and keeps the previous call's contents) and compares every output with the ordinary
 entry point, which is itself checked against the oracle elsewhere.  Collected last on purpose.
