@@ -31,7 +31,7 @@ from paper_2605_14978_b200 import workloads as W
 
 METRIC = "windows/s and logit GB/s (% of B200 HBM peak) at V=128256, K=8, N=2048"
 # DRAM bytes (read + write) per window of the row-reduction kernel from the ncu capture summarised in
-# profiles/row_reduce_bf16_pipe_llama3_like.md (256-window case; traffic grows in proportion to the
+# profiles/row_reduce_pipe_bf16_llama3_like.md (256-window case; traffic grows in proportion to the
 # windows processed).  Only valid for that kernel on that workload shape.
 NCU_TRAFFIC_BYTES_PER_WINDOW = {"llama3_like": 4138559.0}
 NOMINAL_HBM_GBS = 8000.0
@@ -47,6 +47,8 @@ def parse_args():
     ap.add_argument("--workload", default="llama3_like", choices=[w.name for w in W.WORKLOADS])
     ap.add_argument("--mode", default=None, choices=[None, "greedy", "stochastic"])
     ap.add_argument("--windows", type=int, default=None, help="override N (small cases for profiler captures)")
+    ap.add_argument("--logits", default=None, choices=[None, "bf16", "f32"],
+                    help="override the storage type of the logits (same recipe, rounded once to that type)")
     ap.add_argument("--train", action="store_true",
                     help="the step also produces the training-side quantities: KL(Q||P), nabla and the softmax "
                          "normalisers from the scoring pass, the group-relative advantage (groups of 8), and the "
@@ -228,6 +230,9 @@ def run_ppow(args):
     w = W.BY_NAME[args.workload]
     if args.windows:
         w = W.scaled(w, args.windows, name=w.name)
+    if args.logits:
+        import dataclasses
+        w = dataclasses.replace(w, dtype=args.logits)
     mode = args.mode or w.modes[-1]
     bmode = B.PPOW_GREEDY if mode == "greedy" else B.PPOW_STOCHASTIC
     n_chunks = (w.N + W.CHUNK - 1) // W.CHUNK
@@ -357,7 +362,8 @@ def run_ppow(args):
         "logit_gbs": world * algo_bytes / (step_ms * 1e-3) / 1e9,
         "roofline": {"bound": "hbm", "kernel": "row_reduce", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                     "traffic": (NCU_TRAFFIC_BYTES_PER_WINDOW[w.name] * N if w.name in NCU_TRAFFIC_BYTES_PER_WINDOW else None),
+                     "traffic": (NCU_TRAFFIC_BYTES_PER_WINDOW[w.name] * N
+                                 if w.name in NCU_TRAFFIC_BYTES_PER_WINDOW and w.dtype == "bf16" and not args.train else None),
                      "traffic_source": "ncu dram__bytes_read+write on a 256-window capture, scaled by windows",
                      "algorithmic_bytes_per_launch": algo_bytes, "kernel_ms": reduce_avg_ms},
         "training": ({"kl_rev_in_scoring_pass": True, "group_size": group,

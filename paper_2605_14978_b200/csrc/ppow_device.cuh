@@ -141,12 +141,13 @@ struct RowAcc {
         if (REV) B.x = fmaf(eb, xa - xb, B.x);
     }
 
-    // Two packed bf16 pairs: the same operations as two add_pair calls, two per instruction.
+    // Two pairs at once: the same operations as two add_pair calls, on packed f32x2 instructions.
+    // a = two target logits, b = the two draft logits at the same vocabulary entries;
     // s2 = (s, s), nra = (-rho_a, -rho_a), nrb = (-rho_b, -rho_b).
-    __device__ __forceinline__ void add_word(uint32_t wa, uint32_t wb, float2 s2, float2 nra, float2 nrb)
+    __device__ __forceinline__ void add2(float2 a, float2 b, float2 s2, float2 nra, float2 nrb)
     {
-        const float2 xa = __ffma2_rn(make_float2(bf16_lo(wa), bf16_hi(wa)), s2, nra);
-        const float2 xb = __ffma2_rn(make_float2(bf16_lo(wb), bf16_hi(wb)), s2, nrb);
+        const float2 xa = __ffma2_rn(a, s2, nra);
+        const float2 xb = __ffma2_rn(b, s2, nrb);
         const float2 ea = make_float2(ex2_approx(xa.x), ex2_approx(xa.y));
         const float2 eb = make_float2(ex2_approx(xb.x), ex2_approx(xb.y));
         Sa = __fadd2_rn(Sa, ea);
@@ -155,6 +156,12 @@ struct RowAcc {
         const float2 dx = __ffma2_rn(xb, make_float2(-1.0f, -1.0f), xa);   // xa - xb, one rounding
         D = __ffma2_rn(ea, dx, D);
         if (REV) B = __ffma2_rn(eb, dx, B);
+    }
+
+    // One packed bf16 word of each tensor (even entry in the low half).
+    __device__ __forceinline__ void add_word(uint32_t wa, uint32_t wb, float2 s2, float2 nra, float2 nrb)
+    {
+        add2(make_float2(bf16_lo(wa), bf16_hi(wa)), make_float2(bf16_lo(wb), bf16_hi(wb)), s2, nra, nrb);
     }
 
     // Raise the references if this tile's maxima (raw logit units) call for it.

@@ -25,6 +25,7 @@ struct RowJob {
     RowPartial *partials;      // [N*K*segments]
     WsHeader *header;
     int32_t N, K, V;
+    int32_t units_per_row;     // 16-byte units per row (bulk-copy kernel only)
     int32_t segments;          // work items per row
     uint32_t total_items;      // N*K*segments
     float s;                   // log2(e)/T
@@ -89,7 +90,7 @@ __device__ __forceinline__ void open_item(const RowJob &job, ItemCursor &c, uint
     c.u = c.u1 = 0;
     c.pa = c.pb = nullptr;
     if (item >= job.total_items) return;
-    const int32_t units_per_row = job.V >> 3;
+    const int32_t units_per_row = job.units_per_row;
     const uint32_t row = item / (uint32_t)job.segments;
     const int32_t seg = (int32_t)(item % (uint32_t)job.segments);
     c.u = (int32_t)(((int64_t)units_per_row * seg) / job.segments);
@@ -98,51 +99,106 @@ __device__ __forceinline__ void open_item(const RowJob &job, ItemCursor &c, uint
     c.pb = reinterpret_cast<const uint4 *>(job.draft) + (size_t)row * units_per_row;
 }
 
+// Storage formats of the bulk-copy kernel: how a 16-byte unit of logits is read.
+struct FmtBf16 {
+    static constexpr int EPU = 8;   // logits per unit
+    static __device__ __forceinline__ uint4 none()   // a unit that never wins a maximum
+    {
+        return make_uint4(BF16X2_NEG_INF, BF16X2_NEG_INF, BF16X2_NEG_INF, BF16X2_NEG_INF);
+    }
+    static __device__ __forceinline__ float tile_max(const uint4 (&X)[UNROLL])
+    {
+        uint32_t m = max_bf16x2(max_bf16x2(X[0].x, X[0].y), max_bf16x2(X[0].z, X[0].w));
+#pragma unroll
+        for (int j = 1; j < UNROLL; ++j)
+            m = max_bf16x2(m, max_bf16x2(max_bf16x2(X[j].x, X[j].y), max_bf16x2(X[j].z, X[j].w)));
+        return fmaxf(bf16_lo(m), bf16_hi(m));
+    }
+    template <bool REV>
+    static __device__ __forceinline__ void add_unit(RowAcc<REV> &acc, const uint4 &a, const uint4 &b, float2 s2,
+                                                    float2 nra, float2 nrb)
+    {
+        acc.add_word(a.x, b.x, s2, nra, nrb);
+        acc.add_word(a.y, b.y, s2, nra, nrb);
+        acc.add_word(a.z, b.z, s2, nra, nrb);
+        acc.add_word(a.w, b.w, s2, nra, nrb);
+    }
+    // position (0..EPU-1) of the first logit of the unit equal to `value`, or -1
+    static __device__ __forceinline__ int first_equal(const uint4 &w4, float value)
+    {
+        const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+        int pos = -1;
+#pragma unroll
+        for (int q = 3; q >= 0; --q) {
+            if (bf16_hi(w[q]) == value) pos = 2 * q + 1;
+            if (bf16_lo(w[q]) == value) pos = 2 * q;
+        }
+        return pos;
+    }
+};
+
+struct FmtF32 {
+    static constexpr int EPU = 4;
+    static __device__ __forceinline__ uint4 none() { return make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u); }
+    static __device__ __forceinline__ float tile_max(const uint4 (&X)[UNROLL])
+    {
+        float m = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < UNROLL; ++j)
+            m = fmaxf(m, fmaxf(fmaxf(__uint_as_float(X[j].x), __uint_as_float(X[j].y)),
+                               fmaxf(__uint_as_float(X[j].z), __uint_as_float(X[j].w))));
+        return m;
+    }
+    template <bool REV>
+    static __device__ __forceinline__ void add_unit(RowAcc<REV> &acc, const uint4 &a, const uint4 &b, float2 s2,
+                                                    float2 nra, float2 nrb)
+    {
+        acc.add2(make_float2(__uint_as_float(a.x), __uint_as_float(a.y)),
+                 make_float2(__uint_as_float(b.x), __uint_as_float(b.y)), s2, nra, nrb);
+        acc.add2(make_float2(__uint_as_float(a.z), __uint_as_float(a.w)),
+                 make_float2(__uint_as_float(b.z), __uint_as_float(b.w)), s2, nra, nrb);
+    }
+    static __device__ __forceinline__ int first_equal(const uint4 &w4, float value)
+    {
+        int pos = -1;
+        if (__uint_as_float(w4.w) == value) pos = 3;
+        if (__uint_as_float(w4.z) == value) pos = 2;
+        if (__uint_as_float(w4.y) == value) pos = 1;
+        if (__uint_as_float(w4.x) == value) pos = 0;
+        return pos;
+    }
+};
+
 // One tile out of shared memory.  `nu` = units of this lane that exist (UNROLL unless MASKED);
 // refill() is called once every value of the stage sits in registers.
-template <bool MASKED, bool REV, typename Refill>
+template <bool MASKED, bool REV, typename Fmt, typename Refill>
 __device__ __forceinline__ void pipe_tile(const uint4 *sa, const uint4 *sb, int32_t u, int nu, RowAcc<REV> &acc,
                                           float s, Refill refill)
 {
     const int lane = threadIdx.x & 31;
     uint4 A[UNROLL], B[UNROLL];
-    const uint4 none = make_uint4(BF16X2_NEG_INF, BF16X2_NEG_INF, BF16X2_NEG_INF, BF16X2_NEG_INF);
 #pragma unroll
-    for (int j = 0; j < UNROLL; ++j) A[j] = (!MASKED || j < nu) ? sa[j * 32 + lane] : none;
+    for (int j = 0; j < UNROLL; ++j) A[j] = (!MASKED || j < nu) ? sa[j * 32 + lane] : Fmt::none();
 #pragma unroll
-    for (int j = 0; j < UNROLL; ++j) B[j] = (!MASKED || j < nu) ? sb[j * 32 + lane] : none;
+    for (int j = 0; j < UNROLL; ++j) B[j] = (!MASKED || j < nu) ? sb[j * 32 + lane] : Fmt::none();
 
-    uint32_t ma = max_bf16x2(max_bf16x2(A[0].x, A[0].y), max_bf16x2(A[0].z, A[0].w));
-    uint32_t mb = max_bf16x2(max_bf16x2(B[0].x, B[0].y), max_bf16x2(B[0].z, B[0].w));
-#pragma unroll
-    for (int j = 1; j < UNROLL; ++j) {
-        ma = max_bf16x2(ma, max_bf16x2(max_bf16x2(A[j].x, A[j].y), max_bf16x2(A[j].z, A[j].w)));
-        mb = max_bf16x2(mb, max_bf16x2(max_bf16x2(B[j].x, B[j].y), max_bf16x2(B[j].z, B[j].w)));
-    }
-    const float tmax_a = fmaxf(bf16_lo(ma), bf16_hi(ma));
-    const float tmax_b = fmaxf(bf16_lo(mb), bf16_hi(mb));
+    const float tmax_a = Fmt::tile_max(A), tmax_b = Fmt::tile_max(B);
     acc.guard(tmax_a, tmax_b, s);
-    if (tmax_a > acc.max_a) {
+    if (tmax_a > acc.max_a) {   // strict: an equal value seen later has a higher index
         acc.max_a = tmax_a;
-        acc.best = u * 8 + nu;
+        acc.best = u * 8 + nu;  // first unit of this lane in the tile and its unit count, packed
     }
     refill();   // the tile maxima consumed every word of the stage: it may be overwritten now
     const float2 s2 = make_float2(s, s);
     const float2 nra = make_float2(-acc.rho_a, -acc.rho_a), nrb = make_float2(-acc.rho_b, -acc.rho_b);
 #pragma unroll
-    for (int j = 0; j < UNROLL; ++j) {
-        if (!MASKED || j < nu) {
-            acc.add_word(A[j].x, B[j].x, s2, nra, nrb);
-            acc.add_word(A[j].y, B[j].y, s2, nra, nrb);
-            acc.add_word(A[j].z, B[j].z, s2, nra, nrb);
-            acc.add_word(A[j].w, B[j].w, s2, nra, nrb);
-        }
-    }
+    for (int j = 0; j < UNROLL; ++j)
+        if (!MASKED || j < nu) Fmt::add_unit(acc, A[j], B[j], s2, nra, nrb);
     acc.flush();
 }
 
-template <bool REV>
-__global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_bf16_pipe_kernel(const RowJob job)
+template <bool REV, typename Fmt>
+__global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pipe_kernel(const RowJob job)
 {
     extern __shared__ __align__(128) unsigned char pipe_smem[];
     __shared__ __align__(8) uint64_t full_bar[PIPE_WARPS][PIPE_STAGES];
@@ -225,9 +281,9 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_bf1
             produce(st);
         };
         if (n == TILE_UNITS)
-            pipe_tile<false, REV>(sa, sb, C.u + lane, UNROLL, acc, job.s, refill);
+            pipe_tile<false, REV, Fmt>(sa, sb, C.u + lane, UNROLL, acc, job.s, refill);
         else
-            pipe_tile<true, REV>(sa, sb, C.u + lane, min(UNROLL, (n - lane + 31) / 32), acc, job.s, refill);
+            pipe_tile<true, REV, Fmt>(sa, sb, C.u + lane, min(UNROLL, (n - lane + 31) / 32), acc, job.s, refill);
         C.u += n;
 
         if (C.u >= C.u1) {   // end of the item: warp reduction, argmax index, one partial
@@ -238,13 +294,8 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_bf1
             if (my_max == p.max_a) {
                 const int32_t bu = my_best >> 3, bn = my_best & 7;
                 for (int j = 0; j < bn && arg == INT32_MAX; ++j) {
-                    const uint4 w4 = __ldcs(C.pa + bu + j * 32);
-                    const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
-#pragma unroll
-                    for (int q = 3; q >= 0; --q) {
-                        if (bf16_hi(w[q]) == my_max) arg = (bu + j * 32) * 8 + 2 * q + 1;
-                        if (bf16_lo(w[q]) == my_max) arg = (bu + j * 32) * 8 + 2 * q;
-                    }
+                    const int pos = Fmt::first_equal(__ldcs(C.pa + bu + j * 32), my_max);
+                    if (pos >= 0) arg = (bu + j * 32) * Fmt::EPU + pos;
                 }
             }
             arg = warp_min_i32(arg);
@@ -551,9 +602,11 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return PPOW_ERR_CUDA;
 
-    const bool vec_ok = params->dtype == PPOW_BF16 && (params->V % 8 == 0) &&
-                        ((uintptr_t)draft_logits % 16 == 0) && ((uintptr_t)target_logits % 16 == 0) &&
-                        (params->V / 8 >= segments);
+    // the bulk-copy kernel needs rows of whole, 16-byte aligned units; everything else takes the scalar kernel
+    const int epu = params->dtype == PPOW_BF16 ? FmtBf16::EPU : FmtF32::EPU;
+    const bool vec_ok = (params->V % epu == 0) && ((uintptr_t)draft_logits % 16 == 0) &&
+                        ((uintptr_t)target_logits % 16 == 0) && (params->V / epu >= segments);
+    rj.units_per_row = params->V / epu;
     // one warp per work item in every row kernel: a grid that fills the GPU, or fewer CTAs when there is little work.
     // The kernels that also accumulate the sum for KL(Q||P) run only when that output is asked for.
     const bool rev = out->kl_rev != nullptr || out->kl_rev_mean != nullptr;
@@ -561,7 +614,10 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
     int threads = ROW_THREADS;
     size_t dyn_smem = 0;
     if (vec_ok) {
-        kernel = rev ? (const void *)row_reduce_bf16_pipe_kernel<true> : (const void *)row_reduce_bf16_pipe_kernel<false>;
+        if (params->dtype == PPOW_BF16)
+            kernel = rev ? (const void *)row_reduce_pipe_kernel<true, FmtBf16> : (const void *)row_reduce_pipe_kernel<false, FmtBf16>;
+        else
+            kernel = rev ? (const void *)row_reduce_pipe_kernel<true, FmtF32> : (const void *)row_reduce_pipe_kernel<false, FmtF32>;
         threads = PIPE_WARPS * 32;
         dyn_smem = PIPE_SMEM_BYTES;
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PIPE_SMEM_BYTES) != cudaSuccess)

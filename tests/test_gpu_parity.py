@@ -93,7 +93,10 @@ def _both_modes(x, c=0.05, temperature=1.0, eta=1.0, eps=0.5, ref_logp=None):
     (2, 2, 2, torch.float32),           # smallest vocabulary
     (4, 5, 8 * 2333, torch.bfloat16),   # several tiles plus a ragged tail of units
     (1, 8, 128256, torch.bfloat16),     # few rows, large V: rows are split into segments
-    (3, 4, 50000, torch.float32),
+    (3, 4, 50000, torch.float32),       # f32 rows of whole 16-byte units: bulk-copy kernel, rows split into segments
+    (6, 2, 4 * (3 * 512 + 77), torch.float32),   # f32, several tiles plus a ragged tail of units
+    (40, 8, 32000, torch.float32),      # f32, one item per row
+    (2, 3, 4, torch.float32),           # one f32 unit per row
 ])
 def test_shapes_and_paths(N, K, V, dtype):
     x = _random_inputs(N, K, V, dtype, seed=N * 1000 + K * 10 + V % 7)
@@ -125,6 +128,23 @@ def test_unaligned_base_pointer_takes_scalar_path():
         x[key] = flat[1:].view(N, K, V)                            # 2-byte aligned only
         assert x[key].data_ptr() % 16 != 0
     _both_modes(x)
+
+
+def test_f32_unaligned_base_pointer_and_ties():
+    N, K, V = 3, 2, 2048
+    x = _random_inputs(N, K, V, torch.float32, seed=16)
+    t = x["target_logits"]
+    top = t.amax(-1, keepdim=True) + 1.0
+    t[:, :, torch.tensor([2047, 5, 1024, 4], device=DEV)] = top      # exact ties: index 4 wins
+    gpu, ref = _both_modes(x)
+    assert bool((gpu["target_argmax"] == 4).all())
+    for key in ("target_logits", "draft_logits"):
+        flat = torch.empty(N * K * V + 1, dtype=torch.float32, device=DEV)
+        flat[1:].copy_(x[key].flatten())
+        x[key] = flat[1:].view(N, K, V)                              # 4-byte aligned only: scalar kernel
+        assert x[key].data_ptr() % 16 != 0
+    gpu2, _ = _both_modes(x)
+    assert bool((gpu2["target_argmax"] == 4).all())
 
 
 def test_argmax_ties_take_lowest_index():
@@ -193,16 +213,17 @@ def test_extreme_rows_exercise_reference_rebasing():
     _both_modes(x)
 
 
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
 @pytest.mark.parametrize("top", [12.0, 15.5, 16.5, 17.5])
-def test_one_confident_token_over_a_flat_tail(top):
+def test_one_confident_token_over_a_flat_tail(top, dtype):
     """The hardest case for single-precision sums: one term decides the sum and 128255 equal terms, each
     near half an ulp of it, follow.  Every add after the big term rounds the same way, so the error grows
     with the number of adds between two compensated folds; this pins that interval."""
     N, K, V = 4, 8, 128256
     g = torch.Generator(device=DEV).manual_seed(int(top * 10))
     pos = torch.randint(0, V // 8, (N, K), generator=g, device=DEV) * 8      # first logit of a 16-byte unit
-    t = torch.zeros((N, K, V), device=DEV).scatter_(2, pos[..., None], top).to(torch.bfloat16)
-    d = torch.zeros((N, K, V), device=DEV).scatter_(2, pos[..., None], top - 1.0).to(torch.bfloat16)
+    t = torch.zeros((N, K, V), device=DEV).scatter_(2, pos[..., None], top).to(dtype)
+    d = torch.zeros((N, K, V), device=DEV).scatter_(2, pos[..., None], top - 1.0).to(dtype)
     x = {"target_logits": t, "draft_logits": d, "draft_tokens": pos.to(torch.int32),
          "uniforms": torch.rand((N, K), generator=g, device=DEV), "valid_len": None}
     gpu, ref = _both_modes(x, c=0.04)
