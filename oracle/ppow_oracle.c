@@ -29,8 +29,9 @@
  * The training-side quantities at the end of this file (reverse KL, expected acceptance, nabla,
  * group-relative advantage, sliding window scores and the proportional draw of a start) are pinned by
  * tests/test_oracle_training_pins.py.
- * Parity unpinned: Delta with a caller-supplied ref_logp (only its arithmetic is checked; producing
- * ref_logp needs a target model).
+ * Delta with a caller-supplied ref_logp: its arithmetic is pinned, and ppow_oracle_reference_logprob
+ * (end of file) produces ref_logp from the target's logits along its reference window; which logits a
+ * target model would emit there is outside this file.
  */
 #include <math.h>
 #include <pthread.h>
@@ -431,4 +432,33 @@ int32_t ppow_oracle_sample_start(const double *s, int32_t n, double u)
         if (run > thresh) return j;
     }
     return last_positive;   /* rounding left the running sum at or below the threshold */
+}
+
+/* ---- log-probability of the target-preferred reference window (Sec. 4.3.2) ---------------------------
+ * The reference window y is built greedily by the target under its own prefix: y_t = argmax_v
+ * pi_target(v | x, y_<t).  Given the target's logits along that path, ref_logits[n, t, :], its
+ * log-probability is  ref_logp[n] = sum_{t < L_n} max_v log softmax(ref_logits[n,t,:] / T)(v),
+ * and the proximity gap of a drafted window is  Delta = ref_logp[n] - sum_t log P_t(yhat_t). */
+int ppow_oracle_reference_logprob(int32_t N, int32_t K, int32_t V, int32_t dtype, double temperature,
+                                  const void *ref_logits, const int32_t *valid_len, double *ref_logp)
+{
+    if (N < 0 || K < 1 || V < 2 || !(temperature > 0.0)) return 2;
+    if (dtype != ORACLE_F32 && dtype != ORACLE_BF16) return 2;
+    double *buf = (double *)malloc(sizeof(double) * (size_t)V * 3);
+    if (!buf) return 1;
+    double *x = buf, *P = buf + V, *logP = buf + 2 * (size_t)V;
+    for (int32_t n = 0; n < N; ++n) {
+        int32_t L = valid_len ? valid_len[n] : K;
+        if (L < 0) L = 0;
+        if (L > K) L = K;
+        double sum = 0.0;
+        for (int32_t t = 0; t < L; ++t) {
+            size_t row_off = ((size_t)n * K + t) * (size_t)V;
+            int32_t y = row_distribution(ref_logits, dtype, row_off, V, temperature, x, P, logP);
+            sum += logP[y];
+        }
+        ref_logp[n] = sum;
+    }
+    free(buf);
+    return 0;
 }

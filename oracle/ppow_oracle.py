@@ -61,6 +61,8 @@ def _load():
         lib.ppow_oracle_group_advantage.argtypes = [P, ctypes.c_int32, ctypes.c_int32, ctypes.c_double, P]
         lib.ppow_oracle_sliding_scores.restype = ctypes.c_int32
         lib.ppow_oracle_sliding_scores.argtypes = [P, ctypes.c_int32, ctypes.c_int32, P]
+        lib.ppow_oracle_reference_logprob.restype = ctypes.c_int
+        lib.ppow_oracle_reference_logprob.argtypes = [ctypes.c_int32] * 4 + [ctypes.c_double] + [P] * 3
         lib.ppow_oracle_sample_start.restype = ctypes.c_int32
         lib.ppow_oracle_sample_start.argtypes = [P, ctypes.c_int32, ctypes.c_double]
         _lib = lib
@@ -207,3 +209,17 @@ def sample_start(s, u):
     lib = _load()
     s = _np(s, np.float64)
     return int(lib.ppow_oracle_sample_start(_ptr(s) if s.size else None, int(s.shape[0]), float(u)))
+
+
+def reference_logprob(ref_logits, *, temperature=1.0, valid_len=None):
+    """sum_t max_v log softmax(ref_logits[n,t,:]/T) over the valid positions: the target's log-probability of
+    its own greedy reference window (Sec. 4.3.2), given its logits along that window.  float64 [N]."""
+    lib = _load()
+    r, dt = _as_numpy_logits(ref_logits)
+    N, K, V = r.shape
+    vl = _np(valid_len, np.int32)
+    out = np.zeros((N,))
+    rc = lib.ppow_oracle_reference_logprob(N, K, V, dt, float(temperature), _ptr(r), _ptr(vl), _ptr(out))
+    if rc != 0:
+        raise RuntimeError("ppow_oracle_reference_logprob failed with code %d" % rc)
+    return out

@@ -147,3 +147,29 @@ def test_sample_start_is_the_inverse_cdf():
     np.testing.assert_array_equal(draws, np.searchsorted(np.cumsum(w), us * w.sum(), side="right"))
     counts = np.bincount(draws, minlength=12)
     assert sst.chisquare(counts, w / w.sum() * len(us)).pvalue > 1e-4   # drawn in proportion to the weights
+
+
+# ------------------------------------------------------------------ reference-window log-probability (exact Delta)
+
+
+def test_reference_logprob_matches_scipy_and_links_the_two_forms_of_delta():
+    rng = np.random.default_rng(10)
+    d, t, tok = _rand_case(rng, 6, 5, 300)
+    vl = np.array([5, 3, 0, 1, 5, 4], np.int32)
+    for T in (1.0, 0.7):
+        r = oracle.reference_logprob(t, temperature=T, valid_len=vl)
+        lsm = sps.log_softmax(t.astype(np.float64) / T, axis=-1).max(-1)
+        want = np.array([lsm[n, :L].sum() for n, L in enumerate(vl)])
+        np.testing.assert_allclose(r, want, rtol=1e-12, atol=1e-13)
+        assert np.all(r <= 0.0) and r[2] == 0.0
+        # the reference window read off the same logits as the draft is verified on: the exact form of
+        # Delta (Sec. 4.3.2) reduces to the teacher-forced form, position by position
+        a = oracle.score_windows(d, t, tok, mode=oracle.GREEDY, c=0.05, temperature=T, valid_len=vl)
+        b = oracle.score_windows(d, t, tok, mode=oracle.GREEDY, c=0.05, temperature=T, valid_len=vl, ref_logp=r)
+        np.testing.assert_allclose(a["delta"], b["delta"], rtol=1e-11, atol=1e-12)
+        np.testing.assert_array_equal(a["reward_dist"], b["reward_dist"])
+    # a one-hot-like row has log-probability ~0; a uniform row has -ln V
+    u = np.zeros((1, 2, 64), np.float32)
+    u[0, 1, 7] = 80.0
+    r = oracle.reference_logprob(u)
+    assert r[0] == pytest.approx(-math.log(64.0), rel=1e-12)
