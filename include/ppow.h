@@ -206,6 +206,21 @@ ppow_status ppow_expected_acceptance(const ppow_params *params,
                                      const int32_t *valid_len, const float *lse_p, const float *lse_q,
                                      float *expected_accept, void *cuda_stream);
 
+/*
+ * Log-probability of the target-preferred reference window (Sec. 4.3.2): the reference window is built
+ * greedily by the target under its own prefix, y_t = argmax_v pi_target(v | x, y_<t).  Given the target's
+ * logits along that window,
+ *     ref_logp[n] = sum_{t < valid_len[n]} max_v log softmax(ref_target_logits[n,t,:] / T)(v),
+ * which is what ppow_score_windows takes as `ref_logp` to evaluate the proximity gap Delta in its exact
+ * form.  One more streaming pass over one [N,K,V] tensor (params->N, K, V, dtype, temperature are used).
+ *   ref_target_logits   device, [N,K,V] of params->dtype, contiguous
+ *   valid_len           device, [N] int32 or NULL, as for ppow_score_windows
+ *   ref_logp            device, [N] float32 (0 for an empty window)
+ * No workspace.  One thread block per window.
+ */
+ppow_status ppow_reference_logprob(const ppow_params *params, const void *ref_target_logits,
+                                   const int32_t *valid_len, float *ref_logp, void *cuda_stream);
+
 /* Copies the error word that the last ppow_score_windows call on `workspace` left behind into
  * *flags_host (PPOW_FLAG_* bits) and synchronises `cuda_stream` to do so.  Returns
  * PPOW_ERR_DEVICE_TIMEOUT if that bit is set, PPOW_ERR_CUDA on a CUDA failure, else PPOW_OK. */

@@ -25,7 +25,7 @@ EXPORTS = ("ppow_score_workspace_bytes", "ppow_score_windows", "ppow_score_windo
            "ppow_select_workspace_bytes", "ppow_select_windows", "ppow_host_scratch_bytes",
            "ppow_score_and_select_host", "ppow_noalloc_scratch_bytes", "ppow_score_windows_noalloc",
            "ppow_group_advantage", "ppow_sequence_windows", "ppow_expected_acceptance",
-           "ppow_status_string", "ppow_version")
+           "ppow_reference_logprob", "ppow_status_string", "ppow_version")
 
 POSITION_OUTPUTS = {"accept_flag": torch.uint8, "kl": torch.float32, "conf": torch.float32, "crit": torch.float32,
                     "logp_tok": torch.float32, "logq_tok": torch.float32, "target_argmax": torch.int32}
@@ -101,6 +101,8 @@ def load_library():
     lib.ppow_sequence_windows.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
     lib.ppow_expected_acceptance.restype = ctypes.c_int
     lib.ppow_expected_acceptance.argtypes = [ctypes.POINTER(ppow_params), vp, vp, vp, vp, vp, vp, vp]
+    lib.ppow_reference_logprob.restype = ctypes.c_int
+    lib.ppow_reference_logprob.argtypes = [ctypes.POINTER(ppow_params), vp, vp, vp, vp]
     lib.ppow_status_string.restype = ctypes.c_char_p
     lib.ppow_status_string.argtypes = [ctypes.c_int]
     lib.ppow_version.restype = ctypes.c_int
@@ -286,6 +288,16 @@ def ppow_expected_acceptance(params: ppow_params, draft_logits, target_logits, v
         _stream_ptr(stream))
     if st != PPOW_OK:
         raise PpowError(st, "ppow_expected_acceptance")
+
+
+def ppow_reference_logprob(params: ppow_params, ref_target_logits, valid_len, ref_logp, stream=None) -> None:
+    lib = load_library()
+    lt = torch.float32 if params.dtype == PPOW_F32 else torch.bfloat16
+    st = lib.ppow_reference_logprob(ctypes.byref(params), _dev_ptr(ref_target_logits, lt, "ref_target_logits"),
+                                    _dev_ptr(valid_len, torch.int32, "valid_len"),
+                                    _dev_ptr(ref_logp, torch.float32, "ref_logp"), _stream_ptr(stream))
+    if st != PPOW_OK:
+        raise PpowError(st, "ppow_reference_logprob")
 
 
 def _host_ptr(t: Optional[torch.Tensor], dtype=None, name="tensor"):

@@ -251,3 +251,51 @@ def test_expected_acceptance_scalar_path_and_identical_distributions():
     B.ppow_expected_acceptance(params, x["draft_logits"], x["target_logits"], None, gpu["lse_p"], gpu["lse_q"], acc)
     torch.cuda.synchronize()
     np.testing.assert_allclose(acc.cpu().numpy(), 1.0, atol=2e-5)    # min(P, P) sums to 1
+
+
+# ------------------------------------------------------------------ reference-window log-probability (exact Delta)
+
+
+@pytest.mark.parametrize("N,K,V,dtype,T", [(24, 8, 32000, torch.bfloat16, 1.0), (9, 5, 1001, torch.bfloat16, 0.7),
+                                           (6, 3, 5000, torch.float32, 1.3), (3, 10, 151936, torch.bfloat16, 0.7)])
+def test_reference_logprob_matches_oracle_and_feeds_the_exact_delta(N, K, V, dtype, T):
+    g = torch.Generator(device=DEV).manual_seed(N + V)
+    t = (torch.randn((N, K, V), generator=g, device=DEV) * 2.5).to(dtype)
+    d = (t.float() + 0.6 * torch.randn((N, K, V), generator=g, device=DEV)).to(dtype)
+    ref = (t.float() + 0.3 * torch.randn((N, K, V), generator=g, device=DEV)).to(dtype)   # the target on its own path
+    ref[0, 0] = -3.0
+    ref[0, 0, 17] = 40.0                                           # a confident row: log-probability close to 0
+    tok = torch.randint(0, V, (N, K), generator=g, device=DEV, dtype=torch.int32)
+    vl = torch.randint(0, K + 1, (N,), generator=g, device=DEV, dtype=torch.int32)
+    vl[0] = K
+    params = B.make_params(N, K, V, B.PPOW_F32 if dtype == torch.float32 else B.PPOW_BF16, B.PPOW_GREEDY, 0.05, T, 1.0, 6.0)
+    ref_logp = torch.full((N,), 3.0, device=DEV)
+    B.ppow_reference_logprob(params, ref, vl, ref_logp)
+    torch.cuda.synchronize()
+    want = oracle.reference_logprob(ref.cpu(), temperature=T, valid_len=vl.cpu())
+    _assert_close("ref_logp", ref_logp.cpu().numpy(), want)
+    assert bool((ref_logp <= 0).all())
+    # the exact form of Delta end to end: GPU reference log-probability into the GPU scoring pass
+    gpu = B.score_windows(d, t, tok, mode=B.PPOW_GREEDY, c=0.05, temperature=T, eps=6.0, valid_len=vl, ref_logp=ref_logp)
+    torch.cuda.synchronize()
+    o = oracle.score_windows(d.cpu(), t.cpu(), tok.cpu(), mode=oracle.GREEDY, c=0.05, temperature=T, eps=6.0,
+                             valid_len=vl.cpu(), ref_logp=want)
+    _assert_close("delta", gpu["delta"].cpu().numpy(), o["delta"])
+    near = np.abs(o["delta"] - 6.0) < 1e-3
+    np.testing.assert_array_equal(gpu["reward_dist"].cpu().numpy()[~near], o["reward_dist"][~near].astype(np.float32))
+    # reference read off the verification logits themselves: the exact form equals the teacher-forced form
+    B.ppow_reference_logprob(params, t, vl, ref_logp)
+    same = B.score_windows(d, t, tok, mode=B.PPOW_GREEDY, c=0.05, temperature=T, eps=6.0, valid_len=vl, ref_logp=ref_logp)
+    base = B.score_windows(d, t, tok, mode=B.PPOW_GREEDY, c=0.05, temperature=T, eps=6.0, valid_len=vl)
+    torch.cuda.synchronize()
+    _assert_close("delta (two forms)", same["delta"].cpu().numpy(), base["delta"].cpu().numpy().astype(np.float64))
+
+
+def test_reference_logprob_bad_arguments():
+    x = torch.zeros((2, 2, 64), dtype=torch.bfloat16, device=DEV)
+    out = torch.zeros(2, device=DEV)
+    with pytest.raises(B.PpowError):
+        B.ppow_reference_logprob(B.make_params(2, 2, 64, B.PPOW_BF16, 0, 0.05, temperature=0.0), x, None, out)
+    with pytest.raises(B.PpowError):
+        B.ppow_reference_logprob(B.make_params(2, 0, 64, B.PPOW_BF16, 0, 0.05), x, None, out)
+    B.ppow_reference_logprob(B.make_params(0, 2, 64, B.PPOW_BF16, 0, 0.05), x, None, out)     # N = 0: no-op
