@@ -248,13 +248,15 @@ def run_ppow(args):
         out.update(B.alloc_train_outputs(N, K, dev))
         advantage = torch.empty((N,), dtype=torch.float32, device=dev)
         exp_accept = torch.empty((N, K), dtype=torch.float32, device=dev)
+        ref_logp = torch.empty((N,), dtype=torch.float32, device=dev)
+        row_logp = torch.empty((N, K), dtype=torch.float32, device=dev)
         group = 8 if N % 8 == 0 else 1
     ws = B.alloc_workspace(B.ppow_score_workspace_bytes(params), dev)
     selected = torch.empty((n_keep,), dtype=torch.int32, device=dev)
     sel_ws = B.alloc_workspace(B.ppow_select_workspace_bytes(n_total), dev)
     stream = torch.cuda.current_stream()
 
-    acc_events = []
+    acc_events, ref_events = [], []
 
     def step(ev0=None, ev1=None):
         B.ppow_score_windows_traced(params, x["draft_logits"], x["target_logits"], x["draft_tokens"], x["uniforms"],
@@ -269,6 +271,12 @@ def run_ppow(args):
             if ea is not None:
                 eb.record(stream)
                 acc_events.append((ea, eb))
+            # the target's logits stand in for the logits along its reference window (same shape and type)
+            B.ppow_reference_logprob(params, x["target_logits"], x["valid_len"], row_logp, ref_logp, stream)
+            if ea is not None:
+                ec = torch.cuda.Event(enable_timing=True)
+                ec.record(stream)
+                ref_events.append((eb, ec))
         scores = S.gather_scores(out["score"], n_total) if world > 1 else out["score"]   # the one exchange step
         B.ppow_select_windows(scores, n_keep, selected, None, sel_ws, stream)
 
@@ -369,9 +377,12 @@ def run_ppow(args):
         "training": ({"kl_rev_in_scoring_pass": True, "group_size": group,
                       "expected_acceptance_ms": sum(a.elapsed_time(b) for a, b in acc_events) / len(acc_events),
                       "expected_acceptance_gbs": algo_bytes / (sum(a.elapsed_time(b) for a, b in acc_events)
-                                                               / len(acc_events) * 1e-3) / 1e9}
+                                                               / len(acc_events) * 1e-3) / 1e9,
+                      "reference_logprob_ms": sum(a.elapsed_time(b) for a, b in ref_events) / len(ref_events),
+                      "reference_logprob_gbs": 0.5 * algo_bytes / (sum(a.elapsed_time(b) for a, b in ref_events)
+                                                                   / len(ref_events) * 1e-3) / 1e9}
                      if args.train else None),
-        "e2e": e2e, "cpu_baseline": cpu_baseline, "gpu_launches": (5 if args.train else 3) * args.steps, "clocks": clocks,
+        "e2e": e2e, "cpu_baseline": cpu_baseline, "gpu_launches": (7 if args.train else 3) * args.steps, "clocks": clocks,
         "error_flags": flags,
     }
     print(json.dumps(line))

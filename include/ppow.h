@@ -215,11 +215,14 @@ ppow_status ppow_expected_acceptance(const ppow_params *params,
  * form.  One more streaming pass over one [N,K,V] tensor (params->N, K, V, dtype, temperature are used).
  *   ref_target_logits   device, [N,K,V] of params->dtype, contiguous
  *   valid_len           device, [N] int32 or NULL, as for ppow_score_windows
- *   ref_logp            device, [N] float32 (0 for an empty window)
- * No workspace.  One thread block per window.
+ *   row_logp            device, [N,K] float32, required: max_v log softmax(...)(v) per position (0 at
+ *                       positions t >= valid_len[n])
+ *   ref_logp            device, [N] float32 or NULL: the window sums, added in position order (0 for an
+ *                       empty window)
+ * No workspace beyond row_logp.  One thread block per position.
  */
 ppow_status ppow_reference_logprob(const ppow_params *params, const void *ref_target_logits,
-                                   const int32_t *valid_len, float *ref_logp, void *cuda_stream);
+                                   const int32_t *valid_len, float *row_logp, float *ref_logp, void *cuda_stream);
 
 /* Copies the error word that the last ppow_score_windows call on `workspace` left behind into
  * *flags_host (PPOW_FLAG_* bits) and synchronises `cuda_stream` to do so.  Returns

@@ -102,7 +102,7 @@ def load_library():
     lib.ppow_expected_acceptance.restype = ctypes.c_int
     lib.ppow_expected_acceptance.argtypes = [ctypes.POINTER(ppow_params), vp, vp, vp, vp, vp, vp, vp]
     lib.ppow_reference_logprob.restype = ctypes.c_int
-    lib.ppow_reference_logprob.argtypes = [ctypes.POINTER(ppow_params), vp, vp, vp, vp]
+    lib.ppow_reference_logprob.argtypes = [ctypes.POINTER(ppow_params), vp, vp, vp, vp, vp]
     lib.ppow_status_string.restype = ctypes.c_char_p
     lib.ppow_status_string.argtypes = [ctypes.c_int]
     lib.ppow_version.restype = ctypes.c_int
@@ -290,11 +290,12 @@ def ppow_expected_acceptance(params: ppow_params, draft_logits, target_logits, v
         raise PpowError(st, "ppow_expected_acceptance")
 
 
-def ppow_reference_logprob(params: ppow_params, ref_target_logits, valid_len, ref_logp, stream=None) -> None:
+def ppow_reference_logprob(params: ppow_params, ref_target_logits, valid_len, row_logp, ref_logp, stream=None) -> None:
     lib = load_library()
     lt = torch.float32 if params.dtype == PPOW_F32 else torch.bfloat16
     st = lib.ppow_reference_logprob(ctypes.byref(params), _dev_ptr(ref_target_logits, lt, "ref_target_logits"),
                                     _dev_ptr(valid_len, torch.int32, "valid_len"),
+                                    _dev_ptr(row_logp, torch.float32, "row_logp"),
                                     _dev_ptr(ref_logp, torch.float32, "ref_logp"), _stream_ptr(stream))
     if st != PPOW_OK:
         raise PpowError(st, "ppow_reference_logprob")

@@ -203,11 +203,18 @@ __global__ void __launch_bounds__(ACC_THREADS) expected_acceptance_kernel(const 
     }
 }
 
-// ---- log-probability of the reference window: one CTA per window -----------------------------------
+// ---- log-probability of the reference window ---------------------------------------------------------
 // Per row: log2-domain sum of 2^(v*s - rho) against a stale per-thread reference (raised only when a
 // group of logits exceeds it by 2^4), group-local f32 partial folded into a compensated (hi, lo) pair,
 // merged across the block in float64.  log max_v P(v) = ln2 * (M*s - R - log2 S).
 constexpr int REF_THREADS = 256;
+
+__device__ __forceinline__ uint32_t max_bf16x2_(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
 
 struct LseAcc {
     float rho, S, S_hi, S_lo, m;
@@ -239,79 +246,92 @@ struct LseAcc {
     __device__ __forceinline__ void add(float v, float s) { S += ex2f(fmaf(v, s, -rho)); }
 };
 
+// One CTA per (window, position) row from a plain grid; writes log max_v P(v) of the row.
 template <typename T, bool VEC>
-__global__ void __launch_bounds__(REF_THREADS) reference_logprob_kernel(const T *__restrict__ ref,
-                                                                        const int32_t *__restrict__ valid_len, int32_t K,
-                                                                        int32_t V, float s, float *__restrict__ ref_logp)
+__global__ void __launch_bounds__(REF_THREADS) reference_logprob_rows_kernel(const T *__restrict__ ref,
+                                                                             const int32_t *__restrict__ valid_len,
+                                                                             int32_t K, int32_t V, float s,
+                                                                             float *__restrict__ row_logp)
 {
     __shared__ float sh_rho[REF_THREADS / 32], sh_m[REF_THREADS / 32];
     __shared__ double sh_S[REF_THREADS / 32];
-    const int32_t n = (int32_t)blockIdx.x;
+    const size_t row = blockIdx.x;
+    const int32_t n = (int32_t)(row / (size_t)K), k = (int32_t)(row % (size_t)K);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (valid_len && k >= valid_len[n]) {
+        if (tid == 0) row_logp[row] = 0.0f;
+        return;
+    }
+    LseAcc acc;
+    acc.reset();
+    if (VEC) {
+        const uint4 *p = reinterpret_cast<const uint4 *>(ref) + row * (size_t)(V >> 3);
+        const int32_t units = V >> 3;
+        for (int32_t u = tid; u < units; u += 2 * REF_THREADS) {
+            const bool two = u + REF_THREADS < units;
+            const uint4 w0 = __ldcs(p + u);
+            const uint4 w1 = two ? __ldcs(p + u + REF_THREADS) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+            uint32_t mx = max_bf16x2_(max_bf16x2_(max_bf16x2_(w0.x, w0.y), max_bf16x2_(w0.z, w0.w)),
+                                      max_bf16x2_(max_bf16x2_(w1.x, w1.y), max_bf16x2_(w1.z, w1.w)));
+            acc.guard(fmaxf(__uint_as_float(mx << 16), __uint_as_float(mx & 0xffff0000u)), s);
+            const uint32_t w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                if (q < 4 || two) {
+                    acc.add(__uint_as_float(w[q] << 16), s);
+                    acc.add(__uint_as_float(w[q] & 0xffff0000u), s);
+                }
+            }
+            acc.fold();
+        }
+    } else {
+        const T *p = ref + row * (size_t)V;
+        for (int32_t i = tid; i < V; i += REF_THREADS) {
+            const float v = logit_at<T>(p, i);
+            acc.guard(v, s);
+            acc.add(v, s);
+            acc.fold();
+        }
+    }
+    // block merge against the largest reference
+    float R = acc.rho, M = acc.m;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        R = fmaxf(R, __shfl_xor_sync(0xffffffffu, R, o));
+        M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    }
+    const double Sw = warp_sum_double(exp2((double)acc.rho - (double)R) * ((double)acc.S_hi + (double)acc.S_lo));
+    if (lane == 0) {
+        sh_rho[warp] = R;
+        sh_m[warp] = M;
+        sh_S[warp] = Sw;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        float Rb = sh_rho[0], Mb = sh_m[0];
+#pragma unroll
+        for (int i = 1; i < REF_THREADS / 32; ++i) {
+            Rb = fmaxf(Rb, sh_rho[i]);
+            Mb = fmaxf(Mb, sh_m[i]);
+        }
+        double Sb = 0.0;
+#pragma unroll
+        for (int i = 0; i < REF_THREADS / 32; ++i) Sb += exp2((double)sh_rho[i] - (double)Rb) * sh_S[i];
+        row_logp[row] = (float)((fma((double)Mb, (double)s, -(double)Rb) - log2(Sb)) * 0.69314718055994530942);
+    }
+}
+
+// ref_logp[n] = sum of the window's row values, added in position order (float64).
+__global__ void reference_logprob_sum_kernel(const float *__restrict__ row_logp, const int32_t *__restrict__ valid_len,
+                                             int32_t N, int32_t K, float *__restrict__ ref_logp)
+{
+    const int32_t n = (int32_t)(blockIdx.x * blockDim.x + threadIdx.x);
+    if (n >= N) return;
     int32_t L = valid_len ? valid_len[n] : K;
     L = max(0, min(L, K));
-    double window_sum = 0.0;   // thread 0 only
-    for (int32_t t = 0; t < L; ++t) {
-        const size_t row = (size_t)n * K + t;
-        LseAcc acc;
-        acc.reset();
-        if (VEC) {
-            const uint4 *p = reinterpret_cast<const uint4 *>(ref) + row * (size_t)(V >> 3);
-            for (int32_t u = tid; u < (V >> 3); u += REF_THREADS) {
-                const uint4 w4 = __ldcs(p + u);
-                const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
-                float v[8];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    v[2 * q] = __uint_as_float(w[q] << 16);
-                    v[2 * q + 1] = __uint_as_float(w[q] & 0xffff0000u);
-                }
-                float gm = v[0];
-#pragma unroll
-                for (int q = 1; q < 8; ++q) gm = fmaxf(gm, v[q]);
-                acc.guard(gm, s);
-#pragma unroll
-                for (int q = 0; q < 8; ++q) acc.add(v[q], s);
-                acc.fold();
-            }
-        } else {
-            const T *p = ref + row * (size_t)V;
-            for (int32_t i = tid; i < V; i += REF_THREADS) {
-                const float v = logit_at<T>(p, i);
-                acc.guard(v, s);
-                acc.add(v, s);
-                acc.fold();
-            }
-        }
-        // block merge against the largest reference
-        float R = acc.rho, M = acc.m;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            R = fmaxf(R, __shfl_xor_sync(0xffffffffu, R, o));
-            M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-        }
-        const double Sw = warp_sum_double(exp2((double)acc.rho - (double)R) * ((double)acc.S_hi + (double)acc.S_lo));
-        if (lane == 0) {
-            sh_rho[warp] = R;
-            sh_m[warp] = M;
-            sh_S[warp] = Sw;
-        }
-        __syncthreads();
-        if (tid == 0) {
-            float Rb = sh_rho[0], Mb = sh_m[0];
-#pragma unroll
-            for (int i = 1; i < REF_THREADS / 32; ++i) {
-                Rb = fmaxf(Rb, sh_rho[i]);
-                Mb = fmaxf(Mb, sh_m[i]);
-            }
-            double Sb = 0.0;
-#pragma unroll
-            for (int i = 0; i < REF_THREADS / 32; ++i) Sb += exp2((double)sh_rho[i] - (double)Rb) * sh_S[i];
-            window_sum += (fma((double)Mb, (double)s, -(double)Rb) - log2(Sb)) * 0.69314718055994530942;
-        }
-        __syncthreads();
-    }
-    if (tid == 0) ref_logp[n] = (float)window_sum;
+    double sum = 0.0;
+    for (int32_t t = 0; t < L; ++t) sum += (double)row_logp[(size_t)n * K + t];
+    ref_logp[n] = (float)sum;
 }
 
 }  // namespace ppow
@@ -378,27 +398,34 @@ extern "C" ppow_status ppow_expected_acceptance(const ppow_params *params,
 }
 
 extern "C" ppow_status ppow_reference_logprob(const ppow_params *params, const void *ref_target_logits,
-                                              const int32_t *valid_len, float *ref_logp, void *cuda_stream)
+                                              const int32_t *valid_len, float *row_logp, float *ref_logp,
+                                              void *cuda_stream)
 {
     if (!params || params->N < 0 || params->K < 1 || params->V < 2) return PPOW_ERR_INVALID_ARG;
     if (params->dtype != PPOW_F32 && params->dtype != PPOW_BF16) return PPOW_ERR_INVALID_ARG;
     if (!(params->temperature > 0.0f) || !isfinite(params->temperature)) return PPOW_ERR_INVALID_ARG;
     if ((int64_t)params->N * params->K > (int64_t)1 << 26) return PPOW_ERR_INVALID_ARG;
     if (params->N == 0) return PPOW_OK;
-    if (!ref_target_logits || !ref_logp) return PPOW_ERR_INVALID_ARG;
+    if (!ref_target_logits || !row_logp) return PPOW_ERR_INVALID_ARG;
     const size_t esize = params->dtype == PPOW_F32 ? 4 : 2;
     if ((uintptr_t)ref_target_logits % esize) return PPOW_ERR_INVALID_ARG;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     const float s = (float)(1.4426950408889634074 / (double)params->temperature);
-    const unsigned grid = (unsigned)params->N;
+    const unsigned rows = (unsigned)((size_t)params->N * params->K);
     if (params->dtype == PPOW_F32)
-        reference_logprob_kernel<float, false><<<grid, REF_THREADS, 0, stream>>>(
-            (const float *)ref_target_logits, valid_len, params->K, params->V, s, ref_logp);
+        reference_logprob_rows_kernel<float, false><<<rows, REF_THREADS, 0, stream>>>(
+            (const float *)ref_target_logits, valid_len, params->K, params->V, s, row_logp);
     else if (params->V % 8 == 0 && (uintptr_t)ref_target_logits % 16 == 0)
-        reference_logprob_kernel<uint16_t, true><<<grid, REF_THREADS, 0, stream>>>(
-            (const uint16_t *)ref_target_logits, valid_len, params->K, params->V, s, ref_logp);
+        reference_logprob_rows_kernel<uint16_t, true><<<rows, REF_THREADS, 0, stream>>>(
+            (const uint16_t *)ref_target_logits, valid_len, params->K, params->V, s, row_logp);
     else
-        reference_logprob_kernel<uint16_t, false><<<grid, REF_THREADS, 0, stream>>>(
-            (const uint16_t *)ref_target_logits, valid_len, params->K, params->V, s, ref_logp);
-    return cudaGetLastError() == cudaSuccess ? PPOW_OK : PPOW_ERR_CUDA;
+        reference_logprob_rows_kernel<uint16_t, false><<<rows, REF_THREADS, 0, stream>>>(
+            (const uint16_t *)ref_target_logits, valid_len, params->K, params->V, s, row_logp);
+    if (cudaGetLastError() != cudaSuccess) return PPOW_ERR_CUDA;
+    if (ref_logp) {
+        reference_logprob_sum_kernel<<<(unsigned)((params->N + 127) / 128), 128, 0, stream>>>(row_logp, valid_len, params->N,
+                                                                                             params->K, ref_logp);
+        if (cudaGetLastError() != cudaSuccess) return PPOW_ERR_CUDA;
+    }
+    return PPOW_OK;
 }

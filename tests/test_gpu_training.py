@@ -270,11 +270,14 @@ def test_reference_logprob_matches_oracle_and_feeds_the_exact_delta(N, K, V, dty
     vl[0] = K
     params = B.make_params(N, K, V, B.PPOW_F32 if dtype == torch.float32 else B.PPOW_BF16, B.PPOW_GREEDY, 0.05, T, 1.0, 6.0)
     ref_logp = torch.full((N,), 3.0, device=DEV)
-    B.ppow_reference_logprob(params, ref, vl, ref_logp)
+    row_logp = torch.full((N, K), 3.0, device=DEV)
+    B.ppow_reference_logprob(params, ref, vl, row_logp, ref_logp)
     torch.cuda.synchronize()
     want = oracle.reference_logprob(ref.cpu(), temperature=T, valid_len=vl.cpu())
     _assert_close("ref_logp", ref_logp.cpu().numpy(), want)
     assert bool((ref_logp <= 0).all())
+    rows = torch.log_softmax(ref.double() / T, -1).amax(-1) * (torch.arange(K, device=DEV)[None, :] < vl[:, None])
+    _assert_close("row_logp", row_logp.cpu().numpy(), rows.cpu().numpy())
     # the exact form of Delta end to end: GPU reference log-probability into the GPU scoring pass
     gpu = B.score_windows(d, t, tok, mode=B.PPOW_GREEDY, c=0.05, temperature=T, eps=6.0, valid_len=vl, ref_logp=ref_logp)
     torch.cuda.synchronize()
@@ -284,7 +287,7 @@ def test_reference_logprob_matches_oracle_and_feeds_the_exact_delta(N, K, V, dty
     near = np.abs(o["delta"] - 6.0) < 1e-3
     np.testing.assert_array_equal(gpu["reward_dist"].cpu().numpy()[~near], o["reward_dist"][~near].astype(np.float32))
     # reference read off the verification logits themselves: the exact form equals the teacher-forced form
-    B.ppow_reference_logprob(params, t, vl, ref_logp)
+    B.ppow_reference_logprob(params, t, vl, row_logp, ref_logp)
     same = B.score_windows(d, t, tok, mode=B.PPOW_GREEDY, c=0.05, temperature=T, eps=6.0, valid_len=vl, ref_logp=ref_logp)
     base = B.score_windows(d, t, tok, mode=B.PPOW_GREEDY, c=0.05, temperature=T, eps=6.0, valid_len=vl)
     torch.cuda.synchronize()
@@ -293,9 +296,13 @@ def test_reference_logprob_matches_oracle_and_feeds_the_exact_delta(N, K, V, dty
 
 def test_reference_logprob_bad_arguments():
     x = torch.zeros((2, 2, 64), dtype=torch.bfloat16, device=DEV)
-    out = torch.zeros(2, device=DEV)
+    out, rows = torch.zeros(2, device=DEV), torch.zeros((2, 2), device=DEV)
     with pytest.raises(B.PpowError):
-        B.ppow_reference_logprob(B.make_params(2, 2, 64, B.PPOW_BF16, 0, 0.05, temperature=0.0), x, None, out)
+        B.ppow_reference_logprob(B.make_params(2, 2, 64, B.PPOW_BF16, 0, 0.05, temperature=0.0), x, None, rows, out)
     with pytest.raises(B.PpowError):
-        B.ppow_reference_logprob(B.make_params(2, 0, 64, B.PPOW_BF16, 0, 0.05), x, None, out)
-    B.ppow_reference_logprob(B.make_params(0, 2, 64, B.PPOW_BF16, 0, 0.05), x, None, out)     # N = 0: no-op
+        B.ppow_reference_logprob(B.make_params(2, 0, 64, B.PPOW_BF16, 0, 0.05), x, None, rows, out)
+    with pytest.raises(B.PpowError):
+        B.ppow_reference_logprob(B.make_params(2, 2, 64, B.PPOW_BF16, 0, 0.05), x, None, None, out)   # row_logp is required
+    B.ppow_reference_logprob(B.make_params(2, 2, 64, B.PPOW_BF16, 0, 0.05), x, None, rows, None)      # the sums are optional
+    B.ppow_reference_logprob(B.make_params(0, 2, 64, B.PPOW_BF16, 0, 0.05), x, None, rows, out)       # N = 0: no-op
+    torch.cuda.synchronize()
