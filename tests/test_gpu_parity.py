@@ -327,3 +327,29 @@ def test_host_buffer_entry_point_matches_device_path_with_chunking():
         B.ppow_score_and_select_host(params, host["draft_logits"], host["target_logits"], host["draft_tokens"],
                                      host["uniforms"], host["valid_len"], None, out_host, w.n_keep, sel_host, None,
                                      B.alloc_workspace(1024, DEV))
+
+
+def test_randomised_shapes_parameters_and_masks():
+    """Property-style sweep: seeded random shapes (odd and even V, one position to 32, one window to dozens),
+    storage types, temperatures, costs, ragged masks and logit scales; everything is compared with the oracle."""
+    rng = np.random.default_rng(2024)
+    for case in range(40):
+        N = int(rng.integers(1, 40))
+        K = int(rng.choice([1, 2, 3, 5, 8, 10, 12, 17, 32]))
+        V = int(rng.choice([2, 3, 8, 9, 64, 257, 1000, 1024, 4096 + 8, 5000, 20000, 40004]))
+        if N * K * V > 6_000_000:
+            N = max(1, 6_000_000 // (K * V))
+        dtype = torch.bfloat16 if rng.random() < 0.6 else torch.float32
+        T = float(rng.choice([0.5, 0.7, 1.0, 1.7]))
+        c = float(rng.choice([0.0, 0.03, 0.12, 0.5]))
+        scale = float(rng.choice([0.3, 2.0, 8.0]))
+        x = _random_inputs(N, K, V, dtype, seed=1000 + case, sigma=float(rng.choice([0.0, 0.3, 1.5])), scale=scale)
+        if rng.random() < 0.5:
+            x["valid_len"] = torch.from_numpy(rng.integers(0, K + 1, size=N).astype(np.int32)).to(DEV)
+        if rng.random() < 0.3:                                       # drafted tokens that are the target's choice
+            t = x["target_logits"].float()
+            x["draft_tokens"] = torch.where(t == t.amax(-1, keepdim=True), torch.arange(V, device=DEV), V).amin(-1).to(torch.int32)
+        try:
+            _both_modes(x, c=c, temperature=T, eta=float(rng.choice([1.0, 0.4])), eps=float(rng.choice([0.5, 3.0])))
+        except AssertionError as e:
+            raise AssertionError("case %d: N=%d K=%d V=%d %s T=%g c=%g scale=%g: %s" % (case, N, K, V, dtype, T, c, scale, e))
