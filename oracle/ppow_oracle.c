@@ -39,7 +39,7 @@
 #include <stdlib.h>
 #include <string.h>
 
-enum { ORACLE_F32 = 0, ORACLE_BF16 = 1 };
+enum { ORACLE_F32 = 0, ORACLE_BF16 = 1, ORACLE_F16 = 2 };
 enum { ORACLE_GREEDY = 0, ORACLE_STOCHASTIC = 1 };
 
 typedef struct {
@@ -65,10 +65,19 @@ typedef struct {
     int status;
 } oracle_slice;
 
-/* Stored logit -> double; exact for both storage types. */
+/* Stored logit -> double; exact for every storage type. */
 static double load_logit(const void *base, int32_t dtype, size_t idx)
 {
     if (dtype == ORACLE_F32) return (double)((const float *)base)[idx];
+    if (dtype == ORACLE_F16) { /* IEEE binary16: 1 sign, 5 exponent (bias 15), 10 fraction bits */
+        uint16_t h = ((const uint16_t *)base)[idx];
+        int sign = h >> 15, e = (h >> 10) & 31, f = h & 1023;
+        double mag;
+        if (e == 0) mag = ldexp((double)f, -24);                  /* zero and subnormals: f * 2^-24 */
+        else if (e == 31) mag = f ? NAN : INFINITY;
+        else mag = ldexp((double)(1024 + f), e - 25);             /* (1 + f/1024) * 2^(e-15) */
+        return sign ? -mag : mag;
+    }
     uint32_t bits = ((uint32_t)((const uint16_t *)base)[idx]) << 16; /* bf16 = top half of an f32 */
     float f;
     memcpy(&f, &bits, sizeof f);
@@ -211,7 +220,7 @@ int ppow_oracle_score(int32_t N, int32_t K, int32_t V, int32_t dtype, int32_t mo
                       int32_t n_threads)
 {
     if (N < 0 || K < 1 || V < 2 || !(temperature > 0.0) || c < 0.0) return 2;
-    if (dtype != ORACLE_F32 && dtype != ORACLE_BF16) return 2;
+    if (dtype != ORACLE_F32 && dtype != ORACLE_BF16 && dtype != ORACLE_F16) return 2;
     if (mode != ORACLE_GREEDY && mode != ORACLE_STOCHASTIC) return 2;
     if (mode == ORACLE_STOCHASTIC && !uniforms) return 2;
     if (N == 0) return 0;
@@ -360,7 +369,7 @@ int ppow_oracle_diagnostics(int32_t N, int32_t K, int32_t V, int32_t dtype, doub
                             int32_t n_threads)
 {
     if (N < 0 || K < 1 || V < 2 || !(temperature > 0.0)) return 2;
-    if (dtype != ORACLE_F32 && dtype != ORACLE_BF16) return 2;
+    if (dtype != ORACLE_F32 && dtype != ORACLE_BF16 && dtype != ORACLE_F16) return 2;
     if (N == 0) return 0;
     if (n_threads < 1) n_threads = 1;
     if (n_threads > N) n_threads = N;
@@ -443,7 +452,7 @@ int ppow_oracle_reference_logprob(int32_t N, int32_t K, int32_t V, int32_t dtype
                                   const void *ref_logits, const int32_t *valid_len, double *ref_logp)
 {
     if (N < 0 || K < 1 || V < 2 || !(temperature > 0.0)) return 2;
-    if (dtype != ORACLE_F32 && dtype != ORACLE_BF16) return 2;
+    if (dtype != ORACLE_F32 && dtype != ORACLE_BF16 && dtype != ORACLE_F16) return 2;
     double *buf = (double *)malloc(sizeof(double) * (size_t)V * 3);
     if (!buf) return 1;
     double *x = buf, *P = buf + V, *logP = buf + 2 * (size_t)V;
@@ -460,5 +469,13 @@ int ppow_oracle_reference_logprob(int32_t N, int32_t K, int32_t V, int32_t dtype
         ref_logp[n] = sum;
     }
     free(buf);
+    return 0;
+}
+
+/* Decodes n stored logits of the given type to double (used to pin the decoders). */
+int ppow_oracle_decode(const void *stored, int32_t dtype, int64_t n, double *out)
+{
+    if (dtype != ORACLE_F32 && dtype != ORACLE_BF16 && dtype != ORACLE_F16) return 2;
+    for (int64_t i = 0; i < n; ++i) out[i] = load_logit(stored, dtype, (size_t)i);
     return 0;
 }

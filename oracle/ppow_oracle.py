@@ -21,7 +21,7 @@ _LIB = os.path.join(_HERE, "libppow_oracle.so")
 _lock = threading.Lock()
 _lib = None
 
-F32, BF16 = 0, 1
+F32, BF16, F16 = 0, 1, 2
 GREEDY, STOCHASTIC = 0, 1
 
 POSITION_FIELDS = ("accept_flag", "alpha", "entropy", "kl", "conf", "crit", "logp_tok", "logq_tok",
@@ -63,6 +63,8 @@ def _load():
         lib.ppow_oracle_sliding_scores.argtypes = [P, ctypes.c_int32, ctypes.c_int32, P]
         lib.ppow_oracle_reference_logprob.restype = ctypes.c_int
         lib.ppow_oracle_reference_logprob.argtypes = [ctypes.c_int32] * 4 + [ctypes.c_double] + [P] * 3
+        lib.ppow_oracle_decode.restype = ctypes.c_int
+        lib.ppow_oracle_decode.argtypes = [P, ctypes.c_int32, ctypes.c_int64, P]
         lib.ppow_oracle_sample_start.restype = ctypes.c_int32
         lib.ppow_oracle_sample_start.argtypes = [P, ctypes.c_int32, ctypes.c_double]
         _lib = lib
@@ -70,23 +72,25 @@ def _load():
 
 
 def _as_numpy_logits(x):
-    """Accept a numpy float32 / uint16(bf16 bits) array or a CPU torch float32 / bfloat16 tensor."""
+    """Accept a numpy float32 / float16 / uint16 (bf16 bits) array or a CPU torch float32 / bfloat16 / float16 tensor."""
     if not isinstance(x, np.ndarray):
         import torch
         assert isinstance(x, torch.Tensor) and x.device.type == "cpu"
         x = x.contiguous()
         if x.dtype == torch.bfloat16:
             x = x.view(torch.int16).numpy().view(np.uint16)
-        elif x.dtype == torch.float32:
+        elif x.dtype in (torch.float32, torch.float16):
             x = x.numpy()
         else:
-            raise TypeError("logits must be float32 or bfloat16")
+            raise TypeError("logits must be float32, bfloat16 or float16")
     x = np.ascontiguousarray(x)
     if x.dtype == np.float32:
         return x, F32
     if x.dtype == np.uint16:
         return x, BF16
-    raise TypeError("logits must be float32 or uint16 (bf16 bit patterns)")
+    if x.dtype == np.float16:
+        return x.view(np.uint16), F16
+    raise TypeError("logits must be float32, float16 or uint16 (bf16 bit patterns)")
 
 
 def _np(x, dtype):
@@ -222,4 +226,15 @@ def reference_logprob(ref_logits, *, temperature=1.0, valid_len=None):
     rc = lib.ppow_oracle_reference_logprob(N, K, V, dt, float(temperature), _ptr(r), _ptr(vl), _ptr(out))
     if rc != 0:
         raise RuntimeError("ppow_oracle_reference_logprob failed with code %d" % rc)
+    return out
+
+
+def decode(stored):
+    """The oracle's own widening of stored logits to float64 (float32 / float16 arrays, uint16 = bf16 bits)."""
+    lib = _load()
+    a, dt = _as_numpy_logits(stored)
+    out = np.zeros(a.shape, np.float64)
+    rc = lib.ppow_oracle_decode(_ptr(a), dt, int(a.size), _ptr(out))
+    if rc != 0:
+        raise RuntimeError("ppow_oracle_decode failed with code %d" % rc)
     return out

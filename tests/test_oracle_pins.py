@@ -377,3 +377,30 @@ def test_thread_count_does_not_change_results():
     b = oracle.score_windows(d, t, tok, mode=oracle.STOCHASTIC, c=0.05, uniforms=u, n_threads=5)
     for f in a:
         np.testing.assert_array_equal(a[f], b[f])
+
+
+def test_storage_decoders_are_exact_on_every_bit_pattern():
+    bits = np.arange(65536, dtype=np.uint16)
+    half = bits.view(np.float16)
+    finite = np.isfinite(half)
+    got = oracle.decode(half)
+    np.testing.assert_array_equal(got[finite], half[finite].astype(np.float64))          # all 63488 finite halves
+    assert np.all(np.isinf(got[np.isinf(half)])) and np.all(np.isnan(got[np.isnan(half)]))
+    assert np.array_equal(np.signbit(got[finite]), np.signbit(half[finite]))             # -0.0 keeps its sign
+    bf = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
+    want = bf.to(torch.float64).numpy()
+    ok = np.isfinite(want)
+    np.testing.assert_array_equal(oracle.decode(bits)[ok], want[ok])                      # all finite bf16 patterns
+    f = np.array([0.0, -0.0, 1.0, -3.5, 1e-38, 3.4e38, 1.17549435e-38 / 4], np.float32)
+    np.testing.assert_array_equal(oracle.decode(f), f.astype(np.float64))
+
+
+def test_float16_logits_score_like_their_float32_values():
+    rng = np.random.default_rng(41)
+    d, t, tok, u = _rand_case(rng, 4, 3, 200)
+    dh, th = d.astype(np.float16), t.astype(np.float16)
+    a = oracle.score_windows(dh, th, tok, mode=oracle.STOCHASTIC, c=0.05, temperature=0.8, uniforms=u)
+    b = oracle.score_windows(dh.astype(np.float32), th.astype(np.float32), tok, mode=oracle.STOCHASTIC, c=0.05,
+                             temperature=0.8, uniforms=u)
+    for k in a:
+        np.testing.assert_array_equal(a[k], b[k])
