@@ -47,7 +47,7 @@ def parse_args():
     ap.add_argument("--workload", default="llama3_like", choices=[w.name for w in W.WORKLOADS])
     ap.add_argument("--mode", default=None, choices=[None, "greedy", "stochastic"])
     ap.add_argument("--windows", type=int, default=None, help="override N (small cases for profiler captures)")
-    ap.add_argument("--logits", default=None, choices=[None, "bf16", "f32"],
+    ap.add_argument("--logits", default=None, choices=[None, "bf16", "f32", "f16"],
                     help="override the storage type of the logits (same recipe, rounded once to that type)")
     ap.add_argument("--train", action="store_true",
                     help="the step also produces the training-side quantities: KL(Q||P), nabla and the softmax "
@@ -242,7 +242,7 @@ def run_ppow(args):
     N, K, V = w.N, w.K, w.V
     n_total, n_keep = N * world, wg.n_keep
 
-    params = B.make_params(N, K, V, B.PPOW_F32 if w.dtype == "f32" else B.PPOW_BF16, bmode, w.c, w.temperature)
+    params = B.make_params(N, K, V, {"f32": B.PPOW_F32, "bf16": B.PPOW_BF16, "f16": B.PPOW_F16}[w.dtype], bmode, w.c, w.temperature)
     out = B.alloc_outputs(N, K, dev)
     if args.train:
         out.update(B.alloc_train_outputs(N, K, dev))

@@ -43,7 +43,7 @@ typedef enum {
  * `temperature`. */
 typedef enum { PPOW_GREEDY = 0, PPOW_STOCHASTIC = 1 } ppow_mode;
 
-typedef enum { PPOW_F32 = 0, PPOW_BF16 = 1 } ppow_dtype;
+typedef enum { PPOW_F32 = 0, PPOW_BF16 = 1, PPOW_F16 = 2 } ppow_dtype;   /* storage type of the logits */
 
 /* Bits of the device-side error word (ppow_read_error_flags). */
 enum {
@@ -97,7 +97,8 @@ size_t ppow_score_workspace_bytes(const ppow_params *params);
  * Scoring pass (Sec. 4.2 criticality, App. C.1 verification, Sec. 4.3 rewards; Alg. 1 lines
  * "Compute criticality score", "Verify", "proximity gap", reward).
  *
- *   draft_logits, target_logits  device, [N,K,V] of params->dtype, contiguous.  Both tensors are
+ *   draft_logits, target_logits  device, [N,K,V] of params->dtype (float32, bfloat16 or IEEE float16),
+ *                                contiguous.  Both tensors are
  *                                read from HBM exactly once.
  *   draft_tokens                 device, [N,K] int32.  A token outside [0,V) is rejected, gets
  *                                logp_tok = logq_tok = -inf, and sets PPOW_FLAG_TOKEN_RANGE.

@@ -18,7 +18,9 @@ LIB_PATH = os.path.join(_HERE, "libppow.so")
 PPOW_OK = 0
 PPOW_ERR_INVALID_ARG, PPOW_ERR_UNSUPPORTED, PPOW_ERR_WORKSPACE, PPOW_ERR_CUDA, PPOW_ERR_DEVICE_TIMEOUT = 1, 2, 3, 4, 5
 PPOW_GREEDY, PPOW_STOCHASTIC = 0, 1
-PPOW_F32, PPOW_BF16 = 0, 1
+PPOW_F32, PPOW_BF16, PPOW_F16 = 0, 1, 2
+LOGIT_DTYPES = {PPOW_F32: torch.float32, PPOW_BF16: torch.bfloat16, PPOW_F16: torch.float16}
+DTYPE_CODES = {v: k for k, v in LOGIT_DTYPES.items()}
 PPOW_FLAG_TOKEN_RANGE, PPOW_FLAG_DEVICE_TIMEOUT = 1, 2
 
 EXPORTS = ("ppow_score_workspace_bytes", "ppow_score_windows", "ppow_score_windows_traced", "ppow_read_error_flags",
@@ -189,7 +191,7 @@ def ppow_score_windows_traced(params: ppow_params, draft_logits, target_logits, 
                               event_reduce_begin=None, event_reduce_end=None) -> None:
     """ppow_score_windows plus two optional torch.cuda.Event objects recorded around the row-reduction kernel."""
     lib = load_library()
-    lt = torch.float32 if params.dtype == PPOW_F32 else torch.bfloat16
+    lt = LOGIT_DTYPES[params.dtype]
     o = ppow_outputs()
     for name, _ in ppow_outputs._fields_:
         t = outputs.get(name)
@@ -241,7 +243,7 @@ def ppow_score_windows_noalloc(params: ppow_params, draft_logits, target_logits,
     scratch array is used instead.  The binding itself allocates nothing here; ``outputs`` must hold
     preallocated CUDA tensors.  Calls on one device must not overlap (they share the array)."""
     lib = load_library()
-    lt = torch.float32 if params.dtype == PPOW_F32 else torch.bfloat16
+    lt = LOGIT_DTYPES[params.dtype]
     o = ppow_outputs()
     for name, _ in ppow_outputs._fields_:
         want = _ALL_OUTPUTS[name]
@@ -280,7 +282,7 @@ def ppow_sequence_windows(crit, seq_offsets, K: int, scores, uniforms, starts, s
 def ppow_expected_acceptance(params: ppow_params, draft_logits, target_logits, valid_len, lse_p, lse_q,
                              expected_accept, stream=None) -> None:
     lib = load_library()
-    lt = torch.float32 if params.dtype == PPOW_F32 else torch.bfloat16
+    lt = LOGIT_DTYPES[params.dtype]
     st = lib.ppow_expected_acceptance(
         ctypes.byref(params), _dev_ptr(draft_logits, lt, "draft_logits"), _dev_ptr(target_logits, lt, "target_logits"),
         _dev_ptr(valid_len, torch.int32, "valid_len"), _dev_ptr(lse_p, torch.float32, "lse_p"),
@@ -292,7 +294,7 @@ def ppow_expected_acceptance(params: ppow_params, draft_logits, target_logits, v
 
 def ppow_reference_logprob(params: ppow_params, ref_target_logits, valid_len, row_logp, ref_logp, stream=None) -> None:
     lib = load_library()
-    lt = torch.float32 if params.dtype == PPOW_F32 else torch.bfloat16
+    lt = LOGIT_DTYPES[params.dtype]
     st = lib.ppow_reference_logprob(ctypes.byref(params), _dev_ptr(ref_target_logits, lt, "ref_target_logits"),
                                     _dev_ptr(valid_len, torch.int32, "valid_len"),
                                     _dev_ptr(row_logp, torch.float32, "row_logp"),
@@ -320,7 +322,7 @@ def ppow_score_and_select_host(params: ppow_params, draft_logits, target_logits,
                                device_scratch: torch.Tensor, stream=None) -> None:
     """Host-buffer entry point: all tensors except ``device_scratch`` are host tensors (pinned for async copies)."""
     lib = load_library()
-    lt = torch.float32 if params.dtype == PPOW_F32 else torch.bfloat16
+    lt = LOGIT_DTYPES[params.dtype]
     o = ppow_outputs()
     for name, _ in ppow_outputs._fields_:
         want = _ALL_OUTPUTS[name]
@@ -345,7 +347,7 @@ def score_windows(draft_logits, target_logits, draft_tokens, *, mode, c, tempera
     """Allocate outputs and workspace, run ppow_score_windows, return the dict of output tensors
     (with ``train_outputs`` also kl_rev, kl_rev_mean, nabla, lse_p, lse_q)."""
     N, K, V = draft_logits.shape
-    dt = PPOW_F32 if draft_logits.dtype == torch.float32 else PPOW_BF16
+    dt = DTYPE_CODES[draft_logits.dtype]
     params = make_params(N, K, V, dt, mode, c, temperature, eta, eps)
     dev = draft_logits.device
     with torch.cuda.device(dev):

@@ -16,10 +16,17 @@
 // to reach a KL of O(0.01).
 #pragma once
 
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 namespace ppow {
+
+// Storage tags of 16-bit logits: uint16_t stands for bf16 bit patterns, half_bits for IEEE binary16.
+struct half_bits {
+    uint16_t bits;
+};
+__device__ __forceinline__ float f16_to_f32(uint16_t bits) { return __half2float(__ushort_as_half(bits)); }
 
 constexpr float REBASE_LOG2 = 4.0f;      // raise a reference when a tile exceeds it by 2^4
 constexpr float RHO_INIT = -1.0e30f;     // "no reference yet": the first tile always rebases

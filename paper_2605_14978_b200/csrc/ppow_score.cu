@@ -137,6 +137,42 @@ struct FmtBf16 {
     }
 };
 
+struct FmtF16 {
+    static constexpr int EPU = 8;
+    static __device__ __forceinline__ uint4 none() { return make_uint4(0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u); }
+    static __device__ __forceinline__ __half2 h2(uint32_t w) { return *reinterpret_cast<const __half2 *>(&w); }
+    static __device__ __forceinline__ float tile_max(const uint4 (&X)[UNROLL])
+    {
+        __half2 m = __hmax2(__hmax2(h2(X[0].x), h2(X[0].y)), __hmax2(h2(X[0].z), h2(X[0].w)));
+#pragma unroll
+        for (int j = 1; j < UNROLL; ++j)
+            m = __hmax2(m, __hmax2(__hmax2(h2(X[j].x), h2(X[j].y)), __hmax2(h2(X[j].z), h2(X[j].w))));
+        const float2 f = __half22float2(m);
+        return fmaxf(f.x, f.y);
+    }
+    template <bool REV>
+    static __device__ __forceinline__ void add_unit(RowAcc<REV> &acc, const uint4 &a, const uint4 &b, float2 s2,
+                                                    float2 nra, float2 nrb)
+    {
+        acc.add2(__half22float2(h2(a.x)), __half22float2(h2(b.x)), s2, nra, nrb);
+        acc.add2(__half22float2(h2(a.y)), __half22float2(h2(b.y)), s2, nra, nrb);
+        acc.add2(__half22float2(h2(a.z)), __half22float2(h2(b.z)), s2, nra, nrb);
+        acc.add2(__half22float2(h2(a.w)), __half22float2(h2(b.w)), s2, nra, nrb);
+    }
+    static __device__ __forceinline__ int first_equal(const uint4 &w4, float value)
+    {
+        const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+        int pos = -1;
+#pragma unroll
+        for (int q = 3; q >= 0; --q) {
+            const float2 f = __half22float2(h2(w[q]));
+            if (f.y == value) pos = 2 * q + 1;
+            if (f.x == value) pos = 2 * q;
+        }
+        return pos;
+    }
+};
+
 struct FmtF32 {
     static constexpr int EPU = 4;
     static __device__ __forceinline__ uint4 none() { return make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u); }
@@ -324,6 +360,11 @@ __device__ __forceinline__ float load_logit<uint16_t>(const uint16_t *p, size_t 
 {
     return __uint_as_float(((uint32_t)__ldcs(p + i)) << 16);
 }
+template <>
+__device__ __forceinline__ float load_logit<half_bits>(const half_bits *p, size_t i)
+{
+    return f16_to_f32(__ldcs(&p[i].bits));
+}
 
 template <typename T, bool REV>
 __global__ void __launch_bounds__(ROW_THREADS, 4) row_reduce_generic_kernel(const RowJob job)
@@ -384,6 +425,7 @@ struct ScanJob {
 __device__ __forceinline__ double raw_logit(const void *base, int32_t dtype, size_t idx)
 {
     if (dtype == PPOW_F32) return (double)__ldg(reinterpret_cast<const float *>(base) + idx);
+    if (dtype == PPOW_F16) return (double)f16_to_f32(__ldg(reinterpret_cast<const uint16_t *>(base) + idx));
     return (double)__uint_as_float(((uint32_t)__ldg(reinterpret_cast<const uint16_t *>(base) + idx)) << 16);
 }
 
@@ -523,7 +565,7 @@ static bool params_ok(const ppow_params *p)
 {
     if (!p) return false;
     if (p->N < 0 || p->K < 1 || p->V < 2) return false;
-    if (p->dtype != PPOW_F32 && p->dtype != PPOW_BF16) return false;
+    if (p->dtype != PPOW_F32 && p->dtype != PPOW_BF16 && p->dtype != PPOW_F16) return false;
     if (p->mode != PPOW_GREEDY && p->mode != PPOW_STOCHASTIC) return false;
     if (!(p->temperature > 0.0f) || !isfinite(p->temperature)) return false;
     if (!(p->c >= 0.0f) || !isfinite(p->c)) return false;
@@ -603,7 +645,7 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
         return PPOW_ERR_CUDA;
 
     // the bulk-copy kernel needs rows of whole, 16-byte aligned units; everything else takes the scalar kernel
-    const int epu = params->dtype == PPOW_BF16 ? FmtBf16::EPU : FmtF32::EPU;
+    const int epu = params->dtype == PPOW_F32 ? FmtF32::EPU : FmtBf16::EPU;   // 8 logits per unit for both 16-bit types
     const bool vec_ok = (params->V % epu == 0) && ((uintptr_t)draft_logits % 16 == 0) &&
                         ((uintptr_t)target_logits % 16 == 0) && (params->V / epu >= segments);
     rj.units_per_row = params->V / epu;
@@ -616,6 +658,8 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
     if (vec_ok) {
         if (params->dtype == PPOW_BF16)
             kernel = rev ? (const void *)row_reduce_pipe_kernel<true, FmtBf16> : (const void *)row_reduce_pipe_kernel<false, FmtBf16>;
+        else if (params->dtype == PPOW_F16)
+            kernel = rev ? (const void *)row_reduce_pipe_kernel<true, FmtF16> : (const void *)row_reduce_pipe_kernel<false, FmtF16>;
         else
             kernel = rev ? (const void *)row_reduce_pipe_kernel<true, FmtF32> : (const void *)row_reduce_pipe_kernel<false, FmtF32>;
         threads = PIPE_WARPS * 32;
@@ -625,6 +669,9 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
     } else if (params->dtype == PPOW_BF16) {
         kernel = rev ? (const void *)row_reduce_generic_kernel<uint16_t, true>
                      : (const void *)row_reduce_generic_kernel<uint16_t, false>;
+    } else if (params->dtype == PPOW_F16) {
+        kernel = rev ? (const void *)row_reduce_generic_kernel<half_bits, true>
+                     : (const void *)row_reduce_generic_kernel<half_bits, false>;
     } else {
         kernel = rev ? (const void *)row_reduce_generic_kernel<float, true>
                      : (const void *)row_reduce_generic_kernel<float, false>;

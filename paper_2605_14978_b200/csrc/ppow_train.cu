@@ -4,6 +4,7 @@
 // logit tensors a second time.
 #include "../../include/ppow.h"
 
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdint.h>
@@ -146,9 +147,17 @@ __device__ __forceinline__ float logit_at(const T *p, size_t i);
 template <>
 __device__ __forceinline__ float logit_at<float>(const float *p, size_t i) { return __ldcs(p + i); }
 template <>
-__device__ __forceinline__ float logit_at<uint16_t>(const uint16_t *p, size_t i)
+__device__ __forceinline__ float logit_at<uint16_t>(const uint16_t *p, size_t i)   // bf16 bit patterns
 {
     return __uint_as_float(((uint32_t)__ldcs(p + i)) << 16);
+}
+struct half_bits {   // IEEE binary16 bit patterns
+    uint16_t bits;
+};
+template <>
+__device__ __forceinline__ float logit_at<half_bits>(const half_bits *p, size_t i)
+{
+    return __half2float(__ushort_as_half(__ldcs(&p[i].bits)));
 }
 
 // VEC: bf16 rows of whole, 16-byte aligned 8-logit units.
@@ -371,7 +380,7 @@ extern "C" ppow_status ppow_expected_acceptance(const ppow_params *params,
                                                 float *expected_accept, void *cuda_stream)
 {
     if (!params || params->N < 0 || params->K < 1 || params->V < 2) return PPOW_ERR_INVALID_ARG;
-    if (params->dtype != PPOW_F32 && params->dtype != PPOW_BF16) return PPOW_ERR_INVALID_ARG;
+    if (params->dtype != PPOW_F32 && params->dtype != PPOW_BF16 && params->dtype != PPOW_F16) return PPOW_ERR_INVALID_ARG;
     if (!(params->temperature > 0.0f) || !isfinite(params->temperature)) return PPOW_ERR_INVALID_ARG;
     if ((int64_t)params->N * params->K > (int64_t)1 << 26) return PPOW_ERR_INVALID_ARG;
     if (params->N == 0) return PPOW_OK;
@@ -385,6 +394,10 @@ extern "C" ppow_status ppow_expected_acceptance(const ppow_params *params,
     if (params->dtype == PPOW_F32) {
         expected_acceptance_kernel<float, false><<<rows, ACC_THREADS, 0, stream>>>(
             (const float *)target_logits, (const float *)draft_logits, valid_len, lse_p, lse_q, K, V, s, expected_accept);
+    } else if (params->dtype == PPOW_F16) {
+        expected_acceptance_kernel<half_bits, false><<<rows, ACC_THREADS, 0, stream>>>(
+            (const half_bits *)target_logits, (const half_bits *)draft_logits, valid_len, lse_p, lse_q, K, V, s,
+            expected_accept);
     } else if (V % 8 == 0 && (uintptr_t)draft_logits % 16 == 0 && (uintptr_t)target_logits % 16 == 0) {
         expected_acceptance_kernel<uint16_t, true><<<rows, ACC_THREADS, 0, stream>>>(
             (const uint16_t *)target_logits, (const uint16_t *)draft_logits, valid_len, lse_p, lse_q, K, V, s,
@@ -402,7 +415,7 @@ extern "C" ppow_status ppow_reference_logprob(const ppow_params *params, const v
                                               void *cuda_stream)
 {
     if (!params || params->N < 0 || params->K < 1 || params->V < 2) return PPOW_ERR_INVALID_ARG;
-    if (params->dtype != PPOW_F32 && params->dtype != PPOW_BF16) return PPOW_ERR_INVALID_ARG;
+    if (params->dtype != PPOW_F32 && params->dtype != PPOW_BF16 && params->dtype != PPOW_F16) return PPOW_ERR_INVALID_ARG;
     if (!(params->temperature > 0.0f) || !isfinite(params->temperature)) return PPOW_ERR_INVALID_ARG;
     if ((int64_t)params->N * params->K > (int64_t)1 << 26) return PPOW_ERR_INVALID_ARG;
     if (params->N == 0) return PPOW_OK;
@@ -415,6 +428,9 @@ extern "C" ppow_status ppow_reference_logprob(const ppow_params *params, const v
     if (params->dtype == PPOW_F32)
         reference_logprob_rows_kernel<float, false><<<rows, REF_THREADS, 0, stream>>>(
             (const float *)ref_target_logits, valid_len, params->K, params->V, s, row_logp);
+    else if (params->dtype == PPOW_F16)
+        reference_logprob_rows_kernel<half_bits, false><<<rows, REF_THREADS, 0, stream>>>(
+            (const half_bits *)ref_target_logits, valid_len, params->K, params->V, s, row_logp);
     else if (params->V % 8 == 0 && (uintptr_t)ref_target_logits % 16 == 0)
         reference_logprob_rows_kernel<uint16_t, true><<<rows, REF_THREADS, 0, stream>>>(
             (const uint16_t *)ref_target_logits, valid_len, params->K, params->V, s, row_logp);

@@ -33,7 +33,7 @@ class Workload:
     N: int
     K: int
     V: int
-    dtype: str                      # "f32" | "bf16"
+    dtype: str                      # "f32" | "bf16" | "f16"
     noise: str                      # "normal" | "student_t3"
     sigma_lo: float
     sigma_hi: float
@@ -50,7 +50,7 @@ class Workload:
 
     @property
     def torch_dtype(self):
-        return torch.float32 if self.dtype == "f32" else torch.bfloat16
+        return {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[self.dtype]
 
     @property
     def logit_bytes_per_window(self) -> int:

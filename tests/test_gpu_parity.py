@@ -97,6 +97,10 @@ def _both_modes(x, c=0.05, temperature=1.0, eta=1.0, eps=0.5, ref_logp=None):
     (6, 2, 4 * (3 * 512 + 77), torch.float32),   # f32, several tiles plus a ragged tail of units
     (40, 8, 32000, torch.float32),      # f32, one item per row
     (2, 3, 4, torch.float32),           # one f32 unit per row
+    (5, 8, 32000, torch.float16),       # f16: bulk-copy kernel
+    (4, 5, 8 * 2333, torch.float16),    # f16, ragged tail of units
+    (7, 3, 1001, torch.float16),        # f16, scalar kernel
+    (1, 8, 128256, torch.float16),      # f16, rows split into segments
 ])
 def test_shapes_and_paths(N, K, V, dtype):
     x = _random_inputs(N, K, V, dtype, seed=N * 1000 + K * 10 + V % 7)
@@ -128,6 +132,17 @@ def test_unaligned_base_pointer_takes_scalar_path():
         x[key] = flat[1:].view(N, K, V)                            # 2-byte aligned only
         assert x[key].data_ptr() % 16 != 0
     _both_modes(x)
+
+
+def test_float16_workload_and_ties():
+    w = dataclasses.replace(W.scaled(W.WORKLOADS[2], 24), dtype="f16")       # the headline recipe stored as f16
+    x = W.generate(w, DEV)
+    _check_workload(w, x)
+    xt = _random_inputs(3, 2, 4096, torch.float16, seed=18)
+    top = xt["target_logits"].float().amax(-1, keepdim=True) + 1.0
+    xt["target_logits"][:, :, torch.tensor([4095, 9, 2048, 8], device=DEV)] = top.to(torch.float16)
+    gpu, _ = _both_modes(xt)
+    assert bool((gpu["target_argmax"] == 8).all())
 
 
 def test_f32_unaligned_base_pointer_and_ties():
@@ -213,7 +228,7 @@ def test_extreme_rows_exercise_reference_rebasing():
     _both_modes(x)
 
 
-@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32, torch.float16])
 @pytest.mark.parametrize("top", [12.0, 15.5, 16.5, 17.5])
 def test_one_confident_token_over_a_flat_tail(top, dtype):
     """The hardest case for single-precision sums: one term decides the sum and 128255 equal terms, each
@@ -339,7 +354,7 @@ def test_randomised_shapes_parameters_and_masks():
         V = int(rng.choice([2, 3, 8, 9, 64, 257, 1000, 1024, 4096 + 8, 5000, 20000, 40004]))
         if N * K * V > 6_000_000:
             N = max(1, 6_000_000 // (K * V))
-        dtype = torch.bfloat16 if rng.random() < 0.6 else torch.float32
+        dtype = [torch.bfloat16, torch.float32, torch.float16][int(rng.choice(3, p=[0.5, 0.25, 0.25]))]
         T = float(rng.choice([0.5, 0.7, 1.0, 1.7]))
         c = float(rng.choice([0.0, 0.03, 0.12, 0.5]))
         scale = float(rng.choice([0.3, 2.0, 8.0]))

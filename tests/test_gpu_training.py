@@ -85,6 +85,7 @@ def test_reverse_kl_full_size_launch_sampled():
 
 
 @pytest.mark.parametrize("N,K,V,dtype", [(3, 2, 8, torch.bfloat16), (5, 3, 1001, torch.bfloat16), (4, 2, 777, torch.float32),
+                                         (6, 4, 32000, torch.float16), (3, 2, 1001, torch.float16),
                                          (1, 8, 128256, torch.bfloat16), (2, 32, 64, torch.bfloat16)])
 def test_reverse_kl_shapes_and_paths(N, K, V, dtype):
     g = torch.Generator(device=DEV).manual_seed(N * 100 + K)
@@ -225,7 +226,7 @@ def test_expected_acceptance_matches_oracle(idx, n):
     w = W.scaled(W.WORKLOADS[idx], n)
     x = W.generate(w, DEV)
     gpu = _score_with_training_outputs(x, w.modes[-1], w.c, w.temperature)
-    params = B.make_params(w.N, w.K, w.V, B.PPOW_F32 if w.dtype == "f32" else B.PPOW_BF16, 0, w.c, w.temperature)
+    params = B.make_params(w.N, w.K, w.V, B.DTYPE_CODES[w.torch_dtype], 0, w.c, w.temperature)
     acc = torch.full((w.N, w.K), 5.0, device=DEV)
     B.ppow_expected_acceptance(params, x["draft_logits"], x["target_logits"], x["valid_len"], gpu["lse_p"], gpu["lse_q"], acc)
     torch.cuda.synchronize()
@@ -238,6 +239,17 @@ def test_expected_acceptance_matches_oracle(idx, n):
         np.arange(w.K)[None, :] < x["valid_len"].cpu().numpy()[:, None])
     assert np.all((1.0 - a <= np.sqrt(0.5 * kl) + 1e-5)[valid])      # Pinsker (App. B.1)
     assert np.all(a[~valid] == 0.0)
+
+
+def test_expected_acceptance_float16_logits():
+    w = dataclasses.replace(W.scaled(W.WORKLOADS[1], 24), dtype="f16")
+    x = W.generate(w, DEV)
+    gpu = _score_with_training_outputs(x, "greedy", w.c, w.temperature)
+    params = B.make_params(w.N, w.K, w.V, B.PPOW_F16, 0, w.c, w.temperature)
+    acc = torch.empty((w.N, w.K), device=DEV)
+    B.ppow_expected_acceptance(params, x["draft_logits"], x["target_logits"], None, gpu["lse_p"], gpu["lse_q"], acc)
+    torch.cuda.synchronize()
+    _assert_close("expected_accept", acc.cpu().numpy(), _oracle_diag(x, w.temperature)["expected_accept"])
 
 
 def test_expected_acceptance_scalar_path_and_identical_distributions():
@@ -257,7 +269,8 @@ def test_expected_acceptance_scalar_path_and_identical_distributions():
 
 
 @pytest.mark.parametrize("N,K,V,dtype,T", [(24, 8, 32000, torch.bfloat16, 1.0), (9, 5, 1001, torch.bfloat16, 0.7),
-                                           (6, 3, 5000, torch.float32, 1.3), (3, 10, 151936, torch.bfloat16, 0.7)])
+                                           (6, 3, 5000, torch.float32, 1.3), (3, 10, 151936, torch.bfloat16, 0.7),
+                                           (7, 4, 4096, torch.float16, 0.9)])
 def test_reference_logprob_matches_oracle_and_feeds_the_exact_delta(N, K, V, dtype, T):
     g = torch.Generator(device=DEV).manual_seed(N + V)
     t = (torch.randn((N, K, V), generator=g, device=DEV) * 2.5).to(dtype)
@@ -268,7 +281,7 @@ def test_reference_logprob_matches_oracle_and_feeds_the_exact_delta(N, K, V, dty
     tok = torch.randint(0, V, (N, K), generator=g, device=DEV, dtype=torch.int32)
     vl = torch.randint(0, K + 1, (N,), generator=g, device=DEV, dtype=torch.int32)
     vl[0] = K
-    params = B.make_params(N, K, V, B.PPOW_F32 if dtype == torch.float32 else B.PPOW_BF16, B.PPOW_GREEDY, 0.05, T, 1.0, 6.0)
+    params = B.make_params(N, K, V, B.DTYPE_CODES[dtype], B.PPOW_GREEDY, 0.05, T, 1.0, 6.0)
     ref_logp = torch.full((N,), 3.0, device=DEV)
     row_logp = torch.full((N, K), 3.0, device=DEV)
     B.ppow_reference_logprob(params, ref, vl, row_logp, ref_logp)
