@@ -230,6 +230,17 @@ ppow_status ppow_reference_logprob(const ppow_params *params, const void *ref_ta
  * PPOW_ERR_DEVICE_TIMEOUT if that bit is set, PPOW_ERR_CUDA on a CUDA failure, else PPOW_OK. */
 ppow_status ppow_read_error_flags(const void *workspace, uint32_t *flags_host, void *cuda_stream);
 
+/*
+ * Self-test of the device-side failure report.  The scoring kernel's only waits are bounded waits on the
+ * mbarriers of its copy pipeline; when one runs out the kernel sets PPOW_FLAG_DEVICE_TIMEOUT in the
+ * workspace's error word and returns instead of hanging.  This call makes exactly that happen on purpose
+ * and harmlessly: one warp waits, with the same bounded wait, on an mbarrier that nothing completes, for at
+ * most `probes` probes (1..65536), and reports the same way.  Afterwards ppow_read_error_flags(workspace)
+ * returns PPOW_ERR_DEVICE_TIMEOUT with that bit set; the context stays usable.
+ *   workspace   device, >= 256 bytes, 256-byte aligned (its error word is cleared first)
+ */
+ppow_status ppow_selftest_wait_timeout(void *workspace, size_t workspace_bytes, uint32_t probes, void *cuda_stream);
+
 /* Bytes of device scratch ppow_select_windows needs for N scores (0 if N <= 0). */
 size_t ppow_select_workspace_bytes(int32_t N);
 

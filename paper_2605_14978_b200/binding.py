@@ -27,7 +27,7 @@ EXPORTS = ("ppow_score_workspace_bytes", "ppow_score_windows", "ppow_score_windo
            "ppow_select_workspace_bytes", "ppow_select_windows", "ppow_host_scratch_bytes",
            "ppow_score_and_select_host", "ppow_noalloc_scratch_bytes", "ppow_score_windows_noalloc",
            "ppow_group_advantage", "ppow_sequence_windows", "ppow_expected_acceptance",
-           "ppow_reference_logprob", "ppow_status_string", "ppow_version")
+           "ppow_reference_logprob", "ppow_selftest_wait_timeout", "ppow_status_string", "ppow_version")
 
 POSITION_OUTPUTS = {"accept_flag": torch.uint8, "kl": torch.float32, "conf": torch.float32, "crit": torch.float32,
                     "logp_tok": torch.float32, "logq_tok": torch.float32, "target_argmax": torch.int32}
@@ -105,6 +105,8 @@ def load_library():
     lib.ppow_expected_acceptance.argtypes = [ctypes.POINTER(ppow_params), vp, vp, vp, vp, vp, vp, vp]
     lib.ppow_reference_logprob.restype = ctypes.c_int
     lib.ppow_reference_logprob.argtypes = [ctypes.POINTER(ppow_params), vp, vp, vp, vp, vp]
+    lib.ppow_selftest_wait_timeout.restype = ctypes.c_int
+    lib.ppow_selftest_wait_timeout.argtypes = [vp, sz, ctypes.c_uint32, vp]
     lib.ppow_status_string.restype = ctypes.c_char_p
     lib.ppow_status_string.argtypes = [ctypes.c_int]
     lib.ppow_version.restype = ctypes.c_int
@@ -220,6 +222,23 @@ def ppow_read_error_flags(workspace: torch.Tensor, stream=None) -> int:
     if st not in (PPOW_OK, PPOW_ERR_DEVICE_TIMEOUT):
         raise PpowError(st, "ppow_read_error_flags")
     return int(flags.value)
+
+
+def ppow_selftest_wait_timeout(workspace: torch.Tensor, probes: int = 64, stream=None) -> None:
+    """Makes the bounded device-side wait run out on purpose (harmlessly); see include/ppow.h."""
+    lib = load_library()
+    st = lib.ppow_selftest_wait_timeout(_dev_ptr(workspace, torch.uint8, "workspace"), workspace.numel(), int(probes),
+                                        _stream_ptr(stream))
+    if st != PPOW_OK:
+        raise PpowError(st, "ppow_selftest_wait_timeout")
+
+
+def ppow_read_error_status(workspace: torch.Tensor, stream=None):
+    """(status, flags) of ppow_read_error_flags without raising on PPOW_ERR_DEVICE_TIMEOUT."""
+    lib = load_library()
+    flags = ctypes.c_uint32(0)
+    st = lib.ppow_read_error_flags(_dev_ptr(workspace, torch.uint8, "workspace"), ctypes.byref(flags), _stream_ptr(stream))
+    return int(st), int(flags.value)
 
 
 def ppow_select_windows(score, n_keep: int, selected, mask, workspace, stream=None) -> None:

@@ -559,6 +559,23 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
     }
 }
 
+// ---- self-test of the bounded wait ----------------------------------------------------------------
+// One warp waits on an mbarrier that nothing ever completes, with the same bounded wait and the same
+// report as the bulk-copy kernel: the wait runs out, the warp sets PPOW_FLAG_DEVICE_TIMEOUT and returns.
+__global__ void wait_timeout_selftest_kernel(WsHeader *header, uint32_t probes)
+{
+    __shared__ __align__(8) uint64_t bar;
+    const uint32_t bar_addr = smem_addr(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(bar_addr, 1);
+        mbar_init_fence();
+    }
+    __syncwarp();
+    if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_addr, 0u, probes))) {
+        if (threadIdx.x == 0) atomicOr(&header->error_flags, (unsigned)PPOW_FLAG_DEVICE_TIMEOUT);
+    }
+}
+
 // ---- host side ----------------------------------------------------------------------------------
 
 static bool params_ok(const ppow_params *p)
@@ -714,6 +731,17 @@ extern "C" ppow_status ppow_score_windows(const ppow_params *params,
 {
     return ppow_score_windows_traced(params, draft_logits, target_logits, draft_tokens, uniforms, valid_len,
                                      ref_logp, out, workspace, workspace_bytes, cuda_stream, nullptr, nullptr);
+}
+
+extern "C" ppow_status ppow_selftest_wait_timeout(void *workspace, size_t workspace_bytes, uint32_t probes,
+                                                  void *cuda_stream)
+{
+    if (!workspace || ((uintptr_t)workspace % 256) || workspace_bytes < WS_HEADER_BYTES) return PPOW_ERR_WORKSPACE;
+    if (probes < 1 || probes > (1u << 16)) return PPOW_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (cudaMemsetAsync(workspace, 0, WS_HEADER_BYTES, stream) != cudaSuccess) return PPOW_ERR_CUDA;
+    wait_timeout_selftest_kernel<<<1, 32, 0, stream>>>((WsHeader *)workspace, probes);
+    return cudaGetLastError() == cudaSuccess ? PPOW_OK : PPOW_ERR_CUDA;
 }
 
 extern "C" ppow_status ppow_read_error_flags(const void *workspace, uint32_t *flags_host, void *cuda_stream)

@@ -368,3 +368,21 @@ def test_randomised_shapes_parameters_and_masks():
             _both_modes(x, c=c, temperature=T, eta=float(rng.choice([1.0, 0.4])), eps=float(rng.choice([0.5, 3.0])))
         except AssertionError as e:
             raise AssertionError("case %d: N=%d K=%d V=%d %s T=%g c=%g scale=%g: %s" % (case, N, K, V, dtype, T, c, scale, e))
+
+
+def test_bounded_device_wait_reports_a_timeout_and_leaves_the_context_usable():
+    """Failure detection on the device: the copy pipeline's waits are bounded and report through the error
+    word.  The self-test makes such a wait run out (an mbarrier nothing completes) without faulting anything."""
+    ws = B.alloc_workspace(4096, DEV)
+    B.ppow_selftest_wait_timeout(ws, probes=32)
+    status, flags = B.ppow_read_error_status(ws)
+    assert status == B.PPOW_ERR_DEVICE_TIMEOUT and flags & B.PPOW_FLAG_DEVICE_TIMEOUT
+    assert "timeout" in B.ppow_status_string(status).lower() or "wait" in B.ppow_status_string(status).lower()
+    # the context is intact: an ordinary scoring call on the same workspace works and clears the word
+    x = _random_inputs(4, 4, 4096, torch.bfloat16, seed=31)
+    gpu, _ = _both_modes(x)
+    assert B.ppow_read_error_status(gpu["_workspace"]) == (B.PPOW_OK, 0)
+    with pytest.raises(B.PpowError):
+        B.ppow_selftest_wait_timeout(ws, probes=0)
+    with pytest.raises(B.PpowError):
+        B.ppow_selftest_wait_timeout(ws[1:], probes=8)
