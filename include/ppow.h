@@ -30,7 +30,7 @@ extern "C" {
 typedef enum {
     PPOW_OK = 0,
     PPOW_ERR_INVALID_ARG = 1,   /* null/misaligned pointer, size or parameter out of range */
-    PPOW_ERR_UNSUPPORTED = 2,   /* valid request this build cannot serve (e.g. K > 32) */
+    PPOW_ERR_UNSUPPORTED = 2,   /* valid request the library cannot serve (e.g. K > 32) */
     PPOW_ERR_WORKSPACE = 3,     /* workspace missing, misaligned or too small */
     PPOW_ERR_CUDA = 4,          /* a CUDA runtime call or kernel launch failed */
     PPOW_ERR_DEVICE_TIMEOUT = 5 /* a bounded device-side wait gave up (reported by ppow_read_error_flags) */
@@ -38,7 +38,7 @@ typedef enum {
 
 /* Acceptance test.  PPOW_STOCHASTIC is rejection-sampling verification: accept position t iff
  * u_t <= min(1, P_t(yhat_t)/Q_t(yhat_t)) (App. C.1).  PPOW_GREEDY is its temperature-0 decoding
- * case: accept iff yhat_t is the target's most likely token (Sec. 5.1 "Temperatures 0.0 / 1.0";
+ * case: accept iff yhat_t is the target's most likely token (Sec. 5.1, decoding temperatures 0 and 1;
  * Fig. 1).  The mode changes only the acceptance test; entropy, KL and Delta always use
  * `temperature`. */
 typedef enum { PPOW_GREEDY = 0, PPOW_STOCHASTIC = 1 } ppow_mode;
@@ -71,7 +71,7 @@ typedef struct {
     int32_t *accepted_len;   /* [N]   k = number of leading accepted positions (App. C.1, tau) */
     float *reward_speedup;   /* [N]   k/(k*c + 1)                                  (Sec. 4.3.1) */
     float *reward_dist;      /* [N]   eta * 1[k = 0] * 1[Delta < eps]               (Sec. 4.3.2) */
-    float *reward;           /* [N]   reward_speedup + reward_dist                  (Alg. 1, reward line) */
+    float *reward;           /* [N]   reward_speedup + reward_dist                  (Alg. 1, total reward) */
     float *delta;            /* [N]   proximity gap Delta (see ref_logp below)      (Sec. 4.3.2) */
     float *score;            /* [N]   s = mean over valid positions of crit         (Sec. 4.2, s_j) */
     float *kl;               /* [N,K] KL(P_t || Q_t), nats                          (Sec. 4.2) */
@@ -94,12 +94,11 @@ typedef struct {
 size_t ppow_score_workspace_bytes(const ppow_params *params);
 
 /*
- * Scoring pass (Sec. 4.2 criticality, App. C.1 verification, Sec. 4.3 rewards; Alg. 1 lines
- * "Compute criticality score", "Verify", "proximity gap", reward).
+ * Scoring pass (Sec. 4.2 criticality, App. C.1 verification, Sec. 4.3 rewards; the criticality,
+ * verification, proximity-gap and reward steps of Alg. 1).
  *
  *   draft_logits, target_logits  device, [N,K,V] of params->dtype (float32, bfloat16 or IEEE float16),
- *                                contiguous.  Both tensors are
- *                                read from HBM exactly once.
+ *                                contiguous.  Both tensors are read from HBM exactly once.
  *   draft_tokens                 device, [N,K] int32.  A token outside [0,V) is rejected, gets
  *                                logp_tok = logq_tok = -inf, and sets PPOW_FLAG_TOKEN_RANGE.
  *   uniforms                     device, [N,K] float32 in [0,1), drawn by the caller;
@@ -173,7 +172,7 @@ ppow_status ppow_group_advantage(const float *reward, int32_t N, int32_t group_s
                                  float *advantage, void *cuda_stream);
 
 /*
- * Sequence form of Adaptive Divergence-Aware Windowing (Sec. 4.2; Alg. 1 "ADAW-based window selection"):
+ * Sequence form of Adaptive Divergence-Aware Windowing (Sec. 4.2; the window-selection step of Alg. 1):
  * for B responses stored back to back, response b owning positions [seq_offsets[b], seq_offsets[b+1]) of
  * `crit` (the per-position criticality v_t, e.g. the crit output of ppow_score_windows), computes for every
  * start j with a full window inside the response
@@ -260,8 +259,8 @@ ppow_status ppow_select_windows(const float *score, int32_t N, int32_t n_keep,
                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
- * The whole pass for callers whose buffers are in HOST memory (Alg. 1 lines "Compute criticality
- * score" through the reward line, followed by the ADAW ranking of Sec. 4.2): stages the windows
+ * The whole pass for callers whose buffers are in HOST memory (the steps of Alg. 1 from the criticality
+ * score to the reward, followed by the ADAW ranking of Sec. 4.2): stages the windows
  * through `device_scratch` in chunks of as many windows as fit, scores each chunk, keeps the window
  * scores on the device, selects the n_keep best of all N windows and copies every requested result
  * back.  Same arguments as ppow_score_windows + ppow_select_windows except:

@@ -10,7 +10,7 @@
  *   P_t = softmax(target/T), Q_t = softmax(draft/T)                (Sec. 4.2, P_t / Q_t)
  *   H(P_t) = -sum_v P_t(v) log P_t(v)                              (Sec. 4.2, C(P_t))
  *   KL(P_t || Q_t) = sum_v P_t(v) (log P_t(v) - log Q_t(v))        (Sec. 4.2, v_t)
- *   C(P_t) = 1 - H(P_t)/log|V| ,  v_t = C(P_t) * KL(P_t || Q_t)    (Sec. 4.2; Alg. 1 criticality loop)
+ *   C(P_t) = 1 - H(P_t)/log|V| ,  v_t = C(P_t) * KL(P_t || Q_t)    (Sec. 4.2; Alg. 1)
  *   alpha_t = min(1, P_t(yhat_t)/Q_t(yhat_t)), accept iff u_t <= alpha_t   (App. C.1)
  *   greedy (T=0 decoding): accept iff yhat_t == argmax_v P_t(v)    (Sec. 5.1 temperatures; Fig. 1)
  * Per window:
@@ -18,11 +18,11 @@
  *   R_speedup = k/(k*gamma + 1)                                    (Sec. 4.3.1)
  *   Delta = sum_t [log P_t(y_t) - log P_t(yhat_t)], y_t = argmax P_t   (Sec. 4.3.2, teacher-forced reading)
  *        or ref_logp - sum_t log P_t(yhat_t) when the caller supplies the reference window's log-prob
- *   R_dist = eta * 1[k = 0] * 1[Delta < eps]                       (Sec. 4.3.2; Alg. 1 reward line)
- *   r = R_speedup + R_dist                                         (Alg. 1 reward line)
+ *   R_dist = eta * 1[k = 0] * 1[Delta < eps]                       (Sec. 4.3.2; Alg. 1)
+ *   r = R_speedup + R_dist                                         (Alg. 1, total reward)
  *   s = (1/L) sum_t v_t                                            (Sec. 4.2, s_j)
- * Selection: the n_keep windows with the largest s, ties to the lower index (Sec. 4.2, "prioritizes
- * windows with larger s_j").
+ * Selection: the n_keep windows with the largest s, ties to the lower index (Sec. 4.2: ADAW
+ * favours the windows with the larger scores).
  *
  * Pinned by tests/test_oracle_*.py against scipy/torch-float64 library routines, closed forms,
  * the paper's printed reward column and worked examples, brute force and invariants.
@@ -305,7 +305,7 @@ int ppow_oracle_select(const double *score, int32_t N, int32_t n_keep, int32_t *
  *                                                                 (Sec. 4.1); sigma_R is the population standard
  *                                                                 deviation of the group (reading: 1/G, not 1/(G-1))
  *   s_j = (1/K) sum_{t=j}^{j+K-1} v_t,  j = 0..T-K                window scores over one response (Sec. 4.2; Alg. 1)
- *   j* ~ s_j / sum_i s_i                                          Alg. 1 "Sample a training window start"; drawn by
+ *   j* ~ s_j / sum_i s_i                                          Alg. 1, draw of the training window start; drawn by
  *                                                                 inverse CDF from a caller-supplied uniform
  * ===================================================================================== */
 

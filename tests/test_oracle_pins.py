@@ -299,7 +299,7 @@ def test_rewards_delta_and_score_definitions():
         assert (o["delta"][n] == 0) == bool(np.all(tok[n, :Ln] == o["target_argmax"][n, :Ln]))
         want_dist = eta if (k == 0 and o["delta"][n] < eps) else 0.0
         assert o["reward_dist"][n] == want_dist
-        assert o["reward"][n] == pytest.approx(o["reward_speedup"][n] + want_dist)   # Alg. 1 reward line
+        assert o["reward"][n] == pytest.approx(o["reward_speedup"][n] + want_dist)   # Alg. 1: total reward
         assert o["score"][n] == pytest.approx(o["crit"][n, :Ln].mean(), rel=1e-12)   # s = mean of v_t
         assert np.all(o["crit"][n, Ln:] == 0) and np.all(o["accept_flag"][n, Ln:] == 0)
     assert (o["reward_dist"] > 0).any() and (o["reward_dist"] == 0).any()
