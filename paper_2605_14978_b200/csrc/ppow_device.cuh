@@ -34,8 +34,7 @@ constexpr float RHO_INIT = -1.0e30f;     // "no reference yet": the first tile a
 // One partial reduction of (part of) a row; merged later in float64.
 struct __align__(16) RowPartial {
     float rho_a, rho_b;   // references, log2 units
-    float Sa, Sb;         // sums relative to those references (leading parts)
-    float Sa_lo, Sb_lo;   // their compensation terms: the sums are Sa + Sa_lo, Sb + Sb_lo
+    double Sa, Sb;        // sums relative to those references
     double E, D;          // weighted sums relative to the same references
     double B;             // sum 2^x_b (x_a - x_b), for KL(Q||P); 0 unless the call asks for it
     float max_a;          // largest stored target logit seen
@@ -180,32 +179,12 @@ struct RowAcc {
     }
 };
 
-// Error-compensated sum of (hi, lo) pairs across a warp; every lane ends with the same pair.
-__device__ __forceinline__ void warp_sum_pair(float &hi, float &lo)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const float oh = __shfl_xor_sync(0xffffffffu, hi, o);
-        const float ol = __shfl_xor_sync(0xffffffffu, lo, o);
-        const float big = fmaxf(hi, oh), small = fminf(hi, oh);   // sums of 2^x are non-negative
-        const float t = big + small;
-        lo = (lo + ol) + (small - (t - big));
-        hi = t;
-    }
-}
-
+// Maximum over the warp in one instruction (sm_100a reduces f32 min/max in hardware).
 __device__ __forceinline__ float warp_max(float v)
 {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-    return v;
-}
-
-__device__ __forceinline__ float warp_sum(float v)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
+    float r;
+    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+    return r;
 }
 
 __device__ __forceinline__ double warp_sum_f64(double v)
@@ -225,10 +204,8 @@ __device__ __forceinline__ RowPartial warp_reduce(RowAcc<REV> acc)
     RowPartial p;
     p.rho_a = Ra;
     p.rho_b = Rb;
-    warp_sum_pair(acc.Sa_hi, acc.Sa_lo);
-    warp_sum_pair(acc.Sb_hi, acc.Sb_lo);
-    p.Sa = acc.Sa_hi; p.Sa_lo = acc.Sa_lo;
-    p.Sb = acc.Sb_hi; p.Sb_lo = acc.Sb_lo;
+    p.Sa = warp_sum_f64((double)acc.Sa_hi + (double)acc.Sa_lo);
+    p.Sb = warp_sum_f64((double)acc.Sb_hi + (double)acc.Sb_lo);
     p.E = warp_sum_f64((double)acc.E_hi + (double)acc.E_lo);
     p.D = warp_sum_f64((double)acc.D_hi + (double)acc.D_lo);
     p.B = REV ? warp_sum_f64((double)acc.B_hi + (double)acc.B_lo) : 0.0;

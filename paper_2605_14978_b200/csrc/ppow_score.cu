@@ -60,9 +60,9 @@ constexpr uint32_t BF16X2_NEG_INF = 0xff80ff80u;   // packed bf16 (-inf, -inf): 
 
 __device__ __forceinline__ int32_t warp_min_i32(int32_t v)
 {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = min(v, __shfl_xor_sync(0xffffffffu, v, o));
-    return v;
+    int32_t r;
+    asm volatile("redux.sync.min.s32 %0, %1, 0xffffffff;" : "=r"(r) : "r"(v));
+    return r;
 }
 
 // ---- bulk-copy pipeline, one warp per work item (bf16, f16 or f32 rows of whole 16-byte units) -----
@@ -326,15 +326,26 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
         C.u += n;
 
         if (C.u >= C.u1) {   // end of the item: warp reduction, argmax index, one partial
+            // The lanes that hold the item's maximum re-read the units of the tile that raised it, to find the
+            // lowest vocabulary index.  The loads are issued as soon as the maximum is known, so that the rest
+            // of the warp reduction covers their latency.
             const float my_max = acc.max_a;
-            const int32_t my_best = acc.best;
+            const float item_max = warp_max(my_max);
+            const bool holder = my_max == item_max;
+            const int32_t bu = acc.best >> 3, bn = acc.best & 7;
+            uint4 cand[UNROLL];
+#pragma unroll
+            for (int j = 0; j < UNROLL; ++j)
+                if (holder && j < bn) cand[j] = __ldcs(C.pa + bu + j * 32);
             RowPartial p = warp_reduce(acc);
             int32_t arg = INT32_MAX;
-            if (my_max == p.max_a) {
-                const int32_t bu = my_best >> 3, bn = my_best & 7;
-                for (int j = 0; j < bn && arg == INT32_MAX; ++j) {
-                    const int pos = Fmt::first_equal(__ldcs(C.pa + bu + j * 32), my_max);
-                    if (pos >= 0) arg = (bu + j * 32) * Fmt::EPU + pos;
+            if (holder) {
+#pragma unroll
+                for (int j = 0; j < UNROLL; ++j) {
+                    if (j < bn && arg == INT32_MAX) {
+                        const int pos = Fmt::first_equal(cand[j], my_max);
+                        if (pos >= 0) arg = (bu + j * 32) * Fmt::EPU + pos;
+                    }
                 }
             }
             arg = warp_min_i32(arg);
@@ -467,7 +478,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
             const RowPartial p = pp[i];
             const double da = (double)p.rho_a - Ra, db = (double)p.rho_b - Rb;
             const double fa = exp2(da), fb = exp2(db);
-            const double pSa = (double)p.Sa + (double)p.Sa_lo, pSb = (double)p.Sb + (double)p.Sb_lo;
+            const double pSa = p.Sa, pSb = p.Sb;
             const double sa = fa * pSa;
             Sa += sa;
             E += fa * (p.E + da * pSa);
