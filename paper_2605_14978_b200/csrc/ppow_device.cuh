@@ -63,9 +63,11 @@ __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w 
 //
 // A confident distribution puts almost all of a sum into one term: once an f32 accumulator holds
 // that term, every later small term is rounded at its ulp (6e-8 relative each, thousands of times
-// when a lane walks a whole row).  So all four sums are kept as tile-local partials (Sa, Sb, E, D,
-// restarted from zero by flush()) that are folded into running (hi, lo) pairs with an
-// error-compensated add; only the few adds inside one tile can be absorbed.
+// when a lane walks a whole row).  So all sums are kept as tile-local partials (Sa, Sb, E, D, restarted
+// from zero by flush()), and only the few adds inside one tile can be absorbed.  Sa and Sb, which the
+// log-probabilities are read from, are folded into running (hi, lo) pairs with an error-compensated
+// add; for the weighted sums E, D (and B) a plain add per tile measures the same against the float64
+// definition (their tolerance is relative to an entropy or a divergence, not to a log-probability).
 //
 // The tile-local accumulators are float2: lane .x takes the even vocabulary entries of a packed bf16
 // word, lane .y the odd ones, so that the arithmetic runs on sm_100's packed f32x2 instructions
@@ -75,7 +77,8 @@ template <bool REV>
 struct RowAcc {
     float rho_a, rho_b;
     float2 Sa, Sb, E, D, B;
-    float Sa_hi, Sa_lo, Sb_hi, Sb_lo, E_hi, E_lo, D_hi, D_lo, B_hi, B_lo;
+    float Sa_hi, Sa_lo, Sb_hi, Sb_lo;   // compensated running sums of 2^x
+    float Et, Dt, Bt;                   // running weighted sums
     float max_a;
     int32_t best;       // where max_a was first seen (meaning defined by the caller)
 
@@ -83,7 +86,7 @@ struct RowAcc {
     {
         rho_a = rho_b = RHO_INIT;
         Sa = Sb = E = D = B = make_float2(0.0f, 0.0f);
-        Sa_hi = Sa_lo = Sb_hi = Sb_lo = E_hi = E_lo = D_hi = D_lo = B_hi = B_lo = 0.0f;
+        Sa_hi = Sa_lo = Sb_hi = Sb_lo = Et = Dt = Bt = 0.0f;
         max_a = -INFINITY;
         best = 0;
     }
@@ -102,9 +105,9 @@ struct RowAcc {
     {
         two_sum(Sa_hi, Sa_lo, Sa.x + Sa.y);
         two_sum(Sb_hi, Sb_lo, Sb.x + Sb.y);
-        two_sum(E_hi, E_lo, E.x + E.y);
-        two_sum(D_hi, D_lo, D.x + D.y);
-        if (REV) two_sum(B_hi, B_lo, B.x + B.y);
+        Et += E.x + E.y;   // see the note on the struct: a plain add is enough for these three
+        Dt += D.x + D.y;
+        if (REV) Bt += B.x + B.y;
         Sa = Sb = E = D = B = make_float2(0.0f, 0.0f);
     }
 
@@ -118,13 +121,9 @@ struct RowAcc {
         if (da == 0.0f && db == 0.0f) return;
         const float fa = ex2_approx(da), fb = ex2_approx(db);
         const float S = Sa_hi + Sa_lo;
-        E_hi = fa * fmaf(da, S, E_hi + E_lo);
-        D_hi = fa * fmaf(da - db, S, D_hi + D_lo);
-        E_lo = D_lo = 0.0f;
-        if (REV) {
-            B_hi = fb * fmaf(da - db, Sb_hi + Sb_lo, B_hi + B_lo);
-            B_lo = 0.0f;
-        }
+        Et = fa * fmaf(da, S, Et);
+        Dt = fa * fmaf(da - db, S, Dt);
+        if (REV) Bt = fb * fmaf(da - db, Sb_hi + Sb_lo, Bt);
         Sa_hi *= fa;
         Sa_lo *= fa;
         Sb_hi *= fb;
@@ -206,9 +205,9 @@ __device__ __forceinline__ RowPartial warp_reduce(RowAcc<REV> acc)
     p.rho_b = Rb;
     p.Sa = warp_sum_f64((double)acc.Sa_hi + (double)acc.Sa_lo);
     p.Sb = warp_sum_f64((double)acc.Sb_hi + (double)acc.Sb_lo);
-    p.E = warp_sum_f64((double)acc.E_hi + (double)acc.E_lo);
-    p.D = warp_sum_f64((double)acc.D_hi + (double)acc.D_lo);
-    p.B = REV ? warp_sum_f64((double)acc.B_hi + (double)acc.B_lo) : 0.0;
+    p.E = warp_sum_f64((double)acc.Et);
+    p.D = warp_sum_f64((double)acc.Dt);
+    p.B = REV ? warp_sum_f64((double)acc.Bt) : 0.0;
     p.max_a = warp_max(acc.max_a);
     p.argmax = INT32_MAX;
     return p;
