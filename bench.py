@@ -33,7 +33,7 @@ METRIC = "windows/s and logit GB/s (% of B200 HBM peak) at V=128256, K=8, N=2048
 # DRAM bytes (read + write) per window of the row-reduction kernel from the ncu capture summarised in
 # profiles/row_reduce_pipe_bf16_llama3_like.md (256-window case; traffic grows in proportion to the
 # windows processed).  Only valid for that kernel on that workload shape.
-NCU_TRAFFIC_BYTES_PER_WINDOW = {"llama3_like": 4143446.0}
+NCU_TRAFFIC_BYTES_PER_WINDOW = {"llama3_like": 4145686.7}
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
