@@ -307,6 +307,8 @@ int ppow_oracle_select(const double *score, int32_t N, int32_t n_keep, int32_t *
  *   s_j = (1/K) sum_{t=j}^{j+K-1} v_t,  j = 0..T-K                window scores over one response (Sec. 4.2; Alg. 1)
  *   j* ~ s_j / sum_i s_i                                          Alg. 1, draw of the training window start; drawn by
  *                                                                 inverse CDF from a caller-supplied uniform
+ *   j* ~ hard_frac * s_j / sum_i s_i + (1 - hard_frac) / n        hard-window curriculum (App. A): ADAW draw with
+ *                                                                 probability hard_frac, uniform start otherwise
  * ===================================================================================== */
 
 typedef struct {
@@ -441,6 +443,20 @@ int32_t ppow_oracle_sample_start(const double *s, int32_t n, double u)
         if (run > thresh) return j;
     }
     return last_positive;   /* rounding left the running sum at or below the threshold */
+}
+
+/* Hard-window curriculum (App. A, training configuration: the share of ADAW-selected hard windows is
+ * raised 0.2 -> 0.4 -> 0.6 over training; the ablation without ADAW samples windows uniformly).
+ * One start per response: with probability hard_frac it is the ADAW draw above (proportional to s_j),
+ * otherwise a uniform start.  The coin is a caller-supplied uniform u_mix in [0,1): the ADAW branch is
+ * taken iff u_mix < hard_frac, so hard_frac = 0 never takes it and hard_frac = 1 always does; the draw
+ * itself (either branch) uses the second uniform u_draw.  Returns -1 when there is no start. */
+int32_t ppow_oracle_sample_start_mixed(const double *s, int32_t n, double hard_frac, double u_mix, double u_draw)
+{
+    if (n <= 0) return -1;
+    if (u_mix < hard_frac) return ppow_oracle_sample_start(s, n, u_draw);
+    int32_t j = (int32_t)(u_draw * (double)n);
+    return j < n ? j : n - 1;
 }
 
 /* ---- log-probability of the target-preferred reference window (Sec. 4.3.2) ---------------------------

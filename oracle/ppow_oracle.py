@@ -67,6 +67,8 @@ def _load():
         lib.ppow_oracle_decode.argtypes = [P, ctypes.c_int32, ctypes.c_int64, P]
         lib.ppow_oracle_sample_start.restype = ctypes.c_int32
         lib.ppow_oracle_sample_start.argtypes = [P, ctypes.c_int32, ctypes.c_double]
+        lib.ppow_oracle_sample_start_mixed.restype = ctypes.c_int32
+        lib.ppow_oracle_sample_start_mixed.argtypes = [P, ctypes.c_int32] + [ctypes.c_double] * 3
         _lib = lib
     return _lib
 
@@ -213,6 +215,15 @@ def sample_start(s, u):
     lib = _load()
     s = _np(s, np.float64)
     return int(lib.ppow_oracle_sample_start(_ptr(s) if s.size else None, int(s.shape[0]), float(u)))
+
+
+def sample_start_mixed(s, hard_frac, u_mix, u_draw):
+    """Hard-window curriculum draw: the ADAW draw ``sample_start(s, u_draw)`` iff ``u_mix < hard_frac``,
+    otherwise the uniform start ``floor(u_draw * n)`` (-1: no start)."""
+    lib = _load()
+    s = _np(s, np.float64)
+    return int(lib.ppow_oracle_sample_start_mixed(_ptr(s) if s.size else None, int(s.shape[0]), float(hard_frac),
+                                                  float(u_mix), float(u_draw)))
 
 
 def reference_logprob(ref_logits, *, temperature=1.0, valid_len=None):

@@ -149,6 +149,36 @@ def test_sample_start_is_the_inverse_cdf():
     assert sst.chisquare(counts, w / w.sum() * len(us)).pvalue > 1e-4   # drawn in proportion to the weights
 
 
+def test_mixed_draw_reduces_to_its_two_branches_and_mixes_in_the_stated_proportion():
+    # hard-window curriculum (App. A, training configuration): a share hard_frac of the starts comes from the
+    # ADAW draw, the rest is uniform over the starts
+    rng = np.random.default_rng(21)
+    w = rng.random(9) ** 3
+    n = len(w)
+    us = rng.random((30000, 2))
+    # hard_frac = 1: always the ADAW draw, whatever the coin; hard_frac = 0: always floor(u * n)
+    for um, ud in us[:2000]:
+        assert oracle.sample_start_mixed(w, 1.0, um, ud) == oracle.sample_start(w, ud)
+        assert oracle.sample_start_mixed(w, 0.0, um, ud) == int(ud * n)
+    # the coin is strict: u_mix == hard_frac takes the uniform branch, the next float below takes ADAW
+    s = np.array([0.0, 0.0, 0.0, 5.0])
+    assert oracle.sample_start_mixed(s, 0.4, 0.4, 0.1) == 0
+    assert oracle.sample_start_mixed(s, 0.4, np.nextafter(0.4, 0.0), 0.1) == 3
+    assert oracle.sample_start_mixed(np.zeros(0), 0.4, 0.1, 0.1) == -1
+    assert oracle.sample_start_mixed(s, 0.4, 0.9, 0.999999) == 3          # uniform branch reaches the last start
+    # branch by branch against numpy, then the mixture frequencies against hard_frac * w/sum(w) + (1 - hard_frac)/n
+    for hf in (0.2, 0.4, 0.6):                                             # the three stages the paper lists
+        draws = np.array([oracle.sample_start_mixed(w, hf, um, ud) for um, ud in us])
+        adaw = np.searchsorted(np.cumsum(w), us[:, 1] * w.sum(), side="right")
+        unif = np.floor(us[:, 1] * n).astype(int)
+        np.testing.assert_array_equal(draws, np.where(us[:, 0] < hf, adaw, unif))
+        expect = (hf * w / w.sum() + (1.0 - hf) / n) * len(us)
+        assert sst.chisquare(np.bincount(draws, minlength=n), expect).pvalue > 1e-4
+        # and it is NOT either pure branch: the pure-ADAW and pure-uniform frequencies are rejected
+        assert sst.chisquare(np.bincount(draws, minlength=n), w / w.sum() * len(us)).pvalue < 1e-6
+        assert sst.chisquare(np.bincount(draws, minlength=n), np.full(n, len(us) / n)).pvalue < 1e-6
+
+
 # ------------------------------------------------------------------ reference-window log-probability (exact Delta)
 
 
