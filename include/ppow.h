@@ -192,6 +192,23 @@ ppow_status ppow_sequence_windows(const float *crit, const int32_t *seq_offsets,
                                   float *scores, const float *uniforms, int32_t *starts, void *cuda_stream);
 
 /*
+ * ppow_sequence_windows under the hard-window curriculum (App. A, training configuration: the proportion of
+ * ADAW-selected hard windows starts small and is raised over training, 0.2 / 0.4 / 0.6 in the paper's table;
+ * the ablation without ADAW draws windows uniformly).  Scores are as above.  Each response b takes the ADAW
+ * draw (proportional to s_j, from uniforms_draw[b]) iff uniforms_mix[b] < hard_frac, and otherwise the uniform
+ * start floor(uniforms_draw[b] * n_b), n_b = number of starts with a full window.  hard_frac = 1 reproduces
+ * ppow_sequence_windows, hard_frac = 0 is uniform window sampling.  The schedule of hard_frac over training
+ * steps is the caller's.
+ *   hard_frac       in [0,1] (else PPOW_ERR_INVALID_ARG)
+ *   uniforms_mix    device, [B] float32 in [0,1): the per-response coin; required iff starts is given
+ *   uniforms_draw   device, [B] float32 in [0,1): the draw within the chosen branch; required iff starts is given
+ * Everything else as for ppow_sequence_windows.
+ */
+ppow_status ppow_sequence_windows_mixed(const float *crit, const int32_t *seq_offsets, int32_t B, int32_t K,
+                                        float hard_frac, float *scores, const float *uniforms_mix,
+                                        const float *uniforms_draw, int32_t *starts, void *cuda_stream);
+
+/*
  * Expected acceptance probability per position (App. B.1): sum_v min(P_t(v), Q_t(v)) = 1 - TV(P_t, Q_t),
  * the probability that a token drafted from Q_t passes verification.  A second streaming pass over both
  * logit tensors that needs the softmax normalisers of the first: lse_p, lse_q as written by

@@ -26,7 +26,7 @@ PPOW_FLAG_TOKEN_RANGE, PPOW_FLAG_DEVICE_TIMEOUT = 1, 2
 EXPORTS = ("ppow_score_workspace_bytes", "ppow_score_windows", "ppow_score_windows_traced", "ppow_read_error_flags",
            "ppow_select_workspace_bytes", "ppow_select_windows", "ppow_host_scratch_bytes",
            "ppow_score_and_select_host", "ppow_noalloc_scratch_bytes", "ppow_score_windows_noalloc",
-           "ppow_group_advantage", "ppow_sequence_windows", "ppow_expected_acceptance",
+           "ppow_group_advantage", "ppow_sequence_windows", "ppow_sequence_windows_mixed", "ppow_expected_acceptance",
            "ppow_reference_logprob", "ppow_selftest_wait_timeout", "ppow_status_string", "ppow_version")
 
 POSITION_OUTPUTS = {"accept_flag": torch.uint8, "kl": torch.float32, "conf": torch.float32, "crit": torch.float32,
@@ -101,6 +101,8 @@ def load_library():
     lib.ppow_group_advantage.argtypes = [vp, i32, i32, ctypes.c_float, vp, vp]
     lib.ppow_sequence_windows.restype = ctypes.c_int
     lib.ppow_sequence_windows.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
+    lib.ppow_sequence_windows_mixed.restype = ctypes.c_int
+    lib.ppow_sequence_windows_mixed.argtypes = [vp, vp, i32, i32, ctypes.c_float, vp, vp, vp, vp, vp]
     lib.ppow_expected_acceptance.restype = ctypes.c_int
     lib.ppow_expected_acceptance.argtypes = [ctypes.POINTER(ppow_params), vp, vp, vp, vp, vp, vp, vp]
     lib.ppow_reference_logprob.restype = ctypes.c_int
@@ -296,6 +298,19 @@ def ppow_sequence_windows(crit, seq_offsets, K: int, scores, uniforms, starts, s
                                    _stream_ptr(stream))
     if st != PPOW_OK:
         raise PpowError(st, "ppow_sequence_windows")
+
+
+def ppow_sequence_windows_mixed(crit, seq_offsets, K: int, hard_frac: float, scores, uniforms_mix, uniforms_draw,
+                                starts, stream=None) -> None:
+    lib = load_library()
+    B = int(seq_offsets.numel()) - 1 if seq_offsets is not None else 0
+    st = lib.ppow_sequence_windows_mixed(
+        _dev_ptr(crit, torch.float32, "crit"), _dev_ptr(seq_offsets, torch.int32, "seq_offsets"), B, int(K),
+        float(hard_frac), _dev_ptr(scores, torch.float32, "scores"), _dev_ptr(uniforms_mix, torch.float32, "uniforms_mix"),
+        _dev_ptr(uniforms_draw, torch.float32, "uniforms_draw"), _dev_ptr(starts, torch.int32, "starts"),
+        _stream_ptr(stream))
+    if st != PPOW_OK:
+        raise PpowError(st, "ppow_sequence_windows_mixed")
 
 
 def ppow_expected_acceptance(params: ppow_params, draft_logits, target_logits, valid_len, lse_p, lse_q,

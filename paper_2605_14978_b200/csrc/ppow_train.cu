@@ -52,7 +52,8 @@ __global__ void __launch_bounds__(SEQ_THREADS) sequence_windows_kernel(const flo
                                                                        const int32_t *__restrict__ seq_offsets,
                                                                        int32_t K, float *__restrict__ scores,
                                                                        const float *__restrict__ uniforms,
-                                                                       int32_t *__restrict__ starts)
+                                                                       const float *__restrict__ uniforms_mix,
+                                                                       float hard_frac, int32_t *__restrict__ starts)
 {
     __shared__ double chunk[SEQ_THREADS];
     __shared__ double total_sh;
@@ -79,6 +80,16 @@ __global__ void __launch_bounds__(SEQ_THREADS) sequence_windows_kernel(const flo
         if (tid == 0) starts[b] = -1;
         return;
     }
+    const double u = (double)uniforms[b];
+    // hard-window curriculum: the ADAW draw only when the response's coin falls below hard_frac (strictly),
+    // a uniform start otherwise; without a coin array every response takes the ADAW draw
+    if (uniforms_mix && !((double)uniforms_mix[b] < (double)hard_frac)) {
+        if (tid == 0) {
+            const int32_t j = (int32_t)(u * (double)n);
+            starts[b] = j < n ? j : n - 1;
+        }
+        return;
+    }
 
     // pass 1: total of the scores, added in index order
     double run = 0.0;
@@ -98,7 +109,6 @@ __global__ void __launch_bounds__(SEQ_THREADS) sequence_windows_kernel(const flo
     }
     __syncthreads();
     const double total = total_sh;
-    const double u = (double)uniforms[b];
     if (!(total > 0.0)) {   // no signal anywhere: uniform over the starts
         if (tid == 0) {
             const int32_t j = (int32_t)(u * (double)n);
@@ -370,7 +380,22 @@ extern "C" ppow_status ppow_sequence_windows(const float *crit, const int32_t *s
     if (starts && !uniforms) return PPOW_ERR_INVALID_ARG;
     if (!scores && !starts) return PPOW_OK;
     sequence_windows_kernel<<<(unsigned)B, SEQ_THREADS, 0, (cudaStream_t)cuda_stream>>>(crit, seq_offsets, K, scores,
-                                                                                      uniforms, starts);
+                                                                                      uniforms, nullptr, 1.0f, starts);
+    return cudaGetLastError() == cudaSuccess ? PPOW_OK : PPOW_ERR_CUDA;
+}
+
+extern "C" ppow_status ppow_sequence_windows_mixed(const float *crit, const int32_t *seq_offsets, int32_t B, int32_t K,
+                                                   float hard_frac, float *scores, const float *uniforms_mix,
+                                                   const float *uniforms_draw, int32_t *starts, void *cuda_stream)
+{
+    if (B < 0 || K < 1 || K > 1024) return PPOW_ERR_INVALID_ARG;
+    if (!(hard_frac >= 0.0f) || !(hard_frac <= 1.0f)) return PPOW_ERR_INVALID_ARG;
+    if (B == 0) return PPOW_OK;
+    if (!crit || !seq_offsets) return PPOW_ERR_INVALID_ARG;
+    if (starts && (!uniforms_mix || !uniforms_draw)) return PPOW_ERR_INVALID_ARG;
+    if (!scores && !starts) return PPOW_OK;
+    sequence_windows_kernel<<<(unsigned)B, SEQ_THREADS, 0, (cudaStream_t)cuda_stream>>>(
+        crit, seq_offsets, K, scores, uniforms_draw, uniforms_mix, hard_frac, starts);
     return cudaGetLastError() == cudaSuccess ? PPOW_OK : PPOW_ERR_CUDA;
 }
 

@@ -199,6 +199,41 @@ def test_sequence_windows_draw_follows_the_weights():
     assert np.abs(counts / reps - s / s.sum()).max() < 0.03
 
 
+@pytest.mark.parametrize("hard_frac", [0.0, 0.2, 0.4, 0.6, 1.0])
+def test_sequence_windows_mixed_draw_matches_oracle(hard_frac):
+    # hard-window curriculum (App. A): ADAW draw iff the response's coin < hard_frac, uniform start otherwise
+    lengths = [37, 10, 9, 300, 1, 2048, 64, 64, 64, 500, 12, 77] * 6
+    K = 10
+    v, off, u_draw = _sequence_case(lengths, K, seed=int(100 * hard_frac) + 5, zero_seq=1)
+    g = torch.Generator(device=DEV).manual_seed(int(100 * hard_frac) + 6)
+    u_mix = torch.rand(len(lengths), generator=g, device=DEV)
+    if hard_frac < 1.0:                                             # coins live in [0, 1)
+        u_mix[3] = float(np.float32(hard_frac))                     # the coin on the boundary: uniform branch
+    scores = torch.full_like(v, 7.0)
+    starts = torch.full((len(lengths),), -5, dtype=torch.int32, device=DEV)
+    B.ppow_sequence_windows_mixed(v, off, K, hard_frac, scores, u_mix, u_draw, starts)
+    plain_scores, plain_starts = torch.empty_like(v), torch.empty_like(starts)
+    B.ppow_sequence_windows(v, off, K, plain_scores, u_draw, plain_starts)
+    torch.cuda.synchronize()
+    assert torch.equal(scores, plain_scores)                        # the scores do not depend on the curriculum
+    vh, oh = v.cpu().numpy().astype(np.float64), off.cpu().numpy()
+    um, ud = u_mix.cpu().numpy().astype(np.float64), u_draw.cpu().numpy().astype(np.float64)
+    hf = float(np.float32(hard_frac))                               # the value the C ABI carries
+    want = np.array([oracle.sample_start_mixed(oracle.sliding_scores(vh[oh[b]:oh[b + 1]], K), hf, um[b], ud[b])
+                     for b in range(len(lengths))])
+    np.testing.assert_array_equal(starts.cpu().numpy(), want)       # bit-exact
+    if hard_frac == 1.0:
+        assert torch.equal(starts, plain_starts)
+    if 0.0 < hard_frac < 1.0:                                       # both branches were taken
+        took_adaw = um < hf
+        assert took_adaw.any() and (~took_adaw).any()
+    for bad in (-0.1, 1.5, float("nan")):
+        with pytest.raises(B.PpowError):
+            B.ppow_sequence_windows_mixed(v, off, K, bad, scores, u_mix, u_draw, starts)
+    with pytest.raises(B.PpowError):
+        B.ppow_sequence_windows_mixed(v, off, K, 0.5, scores, None, u_draw, starts)
+
+
 def test_sequence_windows_from_scored_positions():
     # criticality of a scored batch, read as one response per window row block
     w = dataclasses.replace(W.scaled(W.WORKLOADS[1], 32), V=4096)
