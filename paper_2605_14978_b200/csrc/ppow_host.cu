@@ -17,7 +17,7 @@ struct ChunkLayout {
     size_t total;
 };
 
-// Device layout of one staged chunk of `cw` windows.
+// Device layout of one staged chunk of `cw` windows out of p->N.
 ChunkLayout chunk_layout(const ppow_params *p, int32_t cw)
 {
     ChunkLayout L;
@@ -36,9 +36,17 @@ ChunkLayout chunk_layout(const ppow_params *p, int32_t cw)
     L.pos_i32 = take(rows * 4);
     L.win_i32 = take((size_t)cw * 4);
     for (int i = 0; i < 5; ++i) L.win_f32[i] = take((size_t)cw * 4);
+    // the workspace serves every chunk the loop will score: full chunks of cw windows and, when cw does not
+    // divide N, a shorter last one -- whose work plan can be finer, hence larger, than a full chunk's
     ppow_params q = *p;
     q.N = cw;
     L.workspace_bytes = ppow_score_workspace_bytes(&q);
+    const int32_t tail = p->N % cw;
+    if (tail > 0) {
+        q.N = tail;
+        const size_t t = ppow_score_workspace_bytes(&q);
+        if (t > L.workspace_bytes) L.workspace_bytes = t;
+    }
     L.workspace = take(L.workspace_bytes);
     L.total = off;
     return L;

@@ -8,11 +8,16 @@
 
 #include <math.h>
 
+#include <atomic>
+
 namespace ppow {
 
 constexpr int ROW_THREADS = 256;   // threads per CTA of the scalar row-reduction kernels
 constexpr int UNROLL = 4;          // 16-byte units per lane per tensor in one tile (< 8: packed with the unit index)
-constexpr int MAX_SEGMENTS = 16;   // a row is split into at most this many work items
+constexpr int TILE_UNITS = 32 * UNROLL;       // 16-byte units per tile per tensor
+constexpr int MAX_SHIFT = 5;       // a row is split into at most 2^5 work items
+constexpr int PLAN_CLASSES = 5;    // row classes of the work plan: items of at most 64, 32, 16, 8, 4 tiles
+constexpr int PLAN_K = 1;          // an item is at most 1/PLAN_K of a resident warp's share of the work still to hand out
 constexpr size_t WS_HEADER_BYTES = 256;
 
 // Workspace header (first WS_HEADER_BYTES of the workspace).
@@ -21,38 +26,106 @@ struct WsHeader {
     unsigned int error_flags;  // PPOW_FLAG_* bits
 };
 
+// Work plan: how the rows are cut into work items.  A row is `tiles` tiles long (a tile is TILE_UNITS
+// 16-byte units of each tensor) and is cut into 2^shift items of whole tiles, item i of a row covering
+// tiles [i*tiles >> shift, (i+1)*tiles >> shift).  Rows come in up to PLAN_CLASSES classes by row index:
+// the first rows are cut into long items (every item ends with a warp reduction), the last rows into
+// short ones, so that the warps, which take items in increasing order from a counter, run out of work
+// at nearly the same time.  Items are numbered class by class, row by row; item i owns partials[i].
+struct WorkPlan {
+    uint32_t item_begin[PLAN_CLASSES + 1];   // first item of each class; [PLAN_CLASSES] = number of items
+    int32_t row_begin[PLAN_CLASSES + 1];     // first row of each class; [PLAN_CLASSES] = N*K
+    int32_t shift[PLAN_CLASSES];             // log2 of the items per row in the class
+    int32_t tiles;                           // tiles per row
+};
+
 struct RowJob {
     const void *target, *draft;
     const int32_t *valid_len;
-    RowPartial *partials;      // [N*K*segments]
+    RowPartial *partials;      // [plan.item_begin[PLAN_CLASSES]]
     WsHeader *header;
+    WorkPlan plan;
     int32_t N, K, V;
     int32_t units_per_row;     // 16-byte units per row (bulk-copy kernel only)
-    int32_t segments;          // work items per row
-    uint32_t total_items;      // N*K*segments
+    int32_t tile_logits;       // logits per tile (scalar kernel: item boundaries in logits)
+    uint32_t total_items;
     float s;                   // log2(e)/T
 };
 
+// (row, first tile, end tile) of a work item
+__device__ __forceinline__ void locate_item(const WorkPlan &plan, uint32_t item, uint32_t &row, int32_t &t0, int32_t &t1)
+{
+    // selects, not indexing: the plan lives in the kernel's parameter space
+    uint32_t ib = plan.item_begin[0];
+    int32_t rb = plan.row_begin[0];
+    int sh = plan.shift[0];
+#pragma unroll
+    for (int c = 1; c < PLAN_CLASSES; ++c) {
+        const bool in = item >= plan.item_begin[c];
+        ib = in ? plan.item_begin[c] : ib;
+        rb = in ? plan.row_begin[c] : rb;
+        sh = in ? plan.shift[c] : sh;
+    }
+    const uint32_t local = item - ib;
+    const uint32_t seg = local & ((1u << sh) - 1u);
+    row = (uint32_t)rb + (local >> sh);
+    t0 = (int32_t)((seg * (uint32_t)plan.tiles) >> sh);
+    t1 = (int32_t)(((seg + 1u) * (uint32_t)plan.tiles) >> sh);
+}
+
+// (first item, number of items) of a row
+__device__ __forceinline__ void row_items(const WorkPlan &plan, uint32_t row, uint32_t &first, int &count)
+{
+    uint32_t ib = plan.item_begin[0];
+    int32_t rb = plan.row_begin[0];
+    int sh = plan.shift[0];
+#pragma unroll
+    for (int c = 1; c < PLAN_CLASSES; ++c) {
+        const bool in = row >= (uint32_t)plan.row_begin[c];
+        ib = in ? plan.item_begin[c] : ib;
+        rb = in ? plan.row_begin[c] : rb;
+        sh = in ? plan.shift[c] : sh;
+    }
+    first = ib + ((row - (uint32_t)rb) << sh);
+    count = 1 << sh;
+}
+
 // ---- work distribution -----------------------------------------------------------------------
-// A work item is one segment of one row, processed by one warp.  Items are handed out by an atomic
-// counter so that ragged windows (rows beyond valid_len are never read), warps that run at different
-// speeds and the tail of the launch stay balanced (a static even split was measured 8 % slower).  Lane 0
-// fetches the id of a warp's next item while the warp is busy with the current one.
+// A work item is one piece of one row, processed by one warp.  Every warp of the launch starts on the
+// item with its own index (no round trip to memory before its first load); all further items are
+// handed out by an atomic counter so that ragged windows (rows beyond valid_len are never read), warps
+// that run at different speeds and the tail of the launch stay balanced (a static even split was
+// measured 8 % slower).  Lane 0 fetches the id of a warp's next item while the warp is busy with the
+// current one.
 
 __device__ __forceinline__ bool item_is_valid(const RowJob &job, uint32_t item)
 {
     if (job.valid_len == nullptr) return true;
-    const uint32_t row = item / (uint32_t)job.segments;
+    uint32_t row;
+    int32_t t0, t1;
+    locate_item(job.plan, item, row, t0, t1);
     const int32_t n = (int32_t)(row / (uint32_t)job.K), k = (int32_t)(row % (uint32_t)job.K);
     return k < __ldg(job.valid_len + n);
 }
 
-__device__ __forceinline__ uint32_t fetch_item(const RowJob &job)
+// Next item from the counter; `workers` = warps of the launch (their first items are not in the counter).
+__device__ __forceinline__ uint32_t fetch_item(const RowJob &job, uint32_t workers)
 {
     uint32_t it;
     do {
-        it = atomicAdd(&job.header->next_item, 1u);
+        it = workers + atomicAdd(&job.header->next_item, 1u);
     } while (it < job.total_items && !item_is_valid(job, it));
+    return it;
+}
+
+// First item of a warp: its own index if that row is valid, else one from the counter (uniform across the warp).
+__device__ __forceinline__ uint32_t first_item(const RowJob &job, uint32_t worker, uint32_t workers, int lane)
+{
+    uint32_t it = worker;
+    if (it < job.total_items && !item_is_valid(job, it)) {
+        if (lane == 0) it = fetch_item(job, workers);
+        it = __shfl_sync(0xffffffffu, it, 0);
+    }
     return it;
 }
 
@@ -75,7 +148,6 @@ __device__ __forceinline__ int32_t warp_min_i32(int32_t v)
 constexpr int PIPE_WARPS = 8;                 // warps per CTA
 constexpr int PIPE_STAGES = 3;                // tiles per warp: one being computed on, two in flight
 constexpr int PIPE_MIN_CTAS = 2;              // 2 CTAs * 8 warps * 3 stages * 4 KB = 192 KB of shared memory per SM
-constexpr int TILE_UNITS = 32 * UNROLL;       // 16-byte units per tile per tensor
 constexpr int TILE_BYTES = TILE_UNITS * 16;   // 2 KB per tensor
 constexpr int ITEM_RING = 8;                  // > PIPE_STAGES + 1 item ids between producer and consumer
 constexpr uint32_t WAIT_LIMIT = 1u << 20;     // probes of one mbarrier before the kernel gives up
@@ -94,10 +166,11 @@ __device__ __forceinline__ void open_item(const RowJob &job, ItemCursor &c, uint
     c.pa = c.pb = nullptr;
     if (item >= job.total_items) return;
     const int32_t units_per_row = job.units_per_row;
-    const uint32_t row = item / (uint32_t)job.segments;
-    const int32_t seg = (int32_t)(item % (uint32_t)job.segments);
-    c.u = (int32_t)(((int64_t)units_per_row * seg) / job.segments);
-    c.u1 = (int32_t)(((int64_t)units_per_row * (seg + 1)) / job.segments);
+    uint32_t row;
+    int32_t t0, t1;
+    locate_item(job.plan, item, row, t0, t1);
+    c.u = t0 * TILE_UNITS;
+    c.u1 = min(t1 * TILE_UNITS, units_per_row);
     c.pa = reinterpret_cast<const uint4 *>(job.target) + (size_t)row * units_per_row;
     c.pb = reinterpret_cast<const uint4 *>(job.draft) + (size_t)row * units_per_row;
 }
@@ -248,30 +321,29 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
     const uint32_t stages_addr = smem_addr(stages);
     const uint32_t bars_addr = smem_addr(&full_bar[warp][0]);
 
+    // the mbarriers of a warp are touched by that warp only (lane 0 arms them and issues the copies, every
+    // lane waits on them): a warp-level barrier after their initialisation is all the set-up needs
     if (lane == 0) {
 #pragma unroll
         for (int st = 0; st < PIPE_STAGES; ++st) mbar_init(bars_addr + 8 * st, 1);
         mbar_init_fence();
     }
-    __syncthreads();
+    __syncwarp();
 
-    // Producer side: P walks the items this warp takes from the work counter and issues one tile per call.
+    // Producer side: P walks the items this warp takes and issues one tile per call.
+    const uint32_t workers = gridDim.x * PIPE_WARPS;
     ItemCursor P, C;
     uint32_t produced = 0, consumed = 0;   // items opened by each side
     uint32_t pending = 0;                   // stages with a copy in flight
-    uint32_t first = 0, upcoming = 0;       // `upcoming` (lane 0): id fetched ahead for the item after P's
-    if (lane == 0) first = fetch_item(job);
-    first = __shfl_sync(0xffffffffu, first, 0);
-    if (lane == 0) {
-        item_ring[warp][0] = first;
-        if (first < job.total_items) upcoming = fetch_item(job);
-    }
+    uint32_t upcoming = 0;                  // (lane 0) id fetched ahead for the item after P's
+    const uint32_t first = first_item(job, blockIdx.x * PIPE_WARPS + warp, workers, lane);
+    if (lane == 0) item_ring[warp][0] = first;
     open_item(job, P, first);
-    open_item(job, C, first);
+    C = P;
     produced = consumed = 1;
 
-    auto produce = [&](int st) {
-        if (P.item >= job.total_items) return;
+    // copies of P's next tile into stage st
+    auto issue = [&](int st) -> int32_t {
         const int32_t n = min(TILE_UNITS, P.u1 - P.u);
         if (lane == 0) {
             const uint32_t bar = bars_addr + 8 * st, dst = stages_addr + st * 2 * TILE_BYTES;
@@ -280,20 +352,34 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
             bulk_load(dst + TILE_BYTES, P.pb + P.u, (uint32_t)n * 16u, bar);
         }
         pending |= 1u << st;
+        return n;
+    };
+    // move P past n units; at the end of its item, on to the item fetched ahead (and fetch the one after)
+    auto advance = [&](int32_t n) {
         P.u += n;
         if (P.u >= P.u1) {
             const uint32_t nx = __shfl_sync(0xffffffffu, upcoming, 0);
             if (lane == 0) {
                 item_ring[warp][produced % ITEM_RING] = nx;
-                if (nx < job.total_items) upcoming = fetch_item(job);
+                if (nx < job.total_items) upcoming = fetch_item(job, workers);
             }
             ++produced;
             open_item(job, P, nx);
         }
     };
+    auto produce = [&](int st) {
+        if (P.item >= job.total_items) return;
+        advance(issue(st));
+    };
 
+    // the first tile is on its way before the warp's first visit to the work counter
+    if (P.item < job.total_items) {
+        const int32_t n = issue(0);
+        if (lane == 0) upcoming = fetch_item(job, workers);
+        advance(n);
+    }
 #pragma unroll
-    for (int st = 0; st < PIPE_STAGES; ++st) produce(st);
+    for (int st = 1; st < PIPE_STAGES; ++st) produce(st);
 
     uint32_t phases = 0;
     int st = 0;
@@ -338,6 +424,13 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
             for (int j = 0; j < UNROLL; ++j)
                 if (holder && j < bn) cand[j] = __ldcs(C.pa + bu + j * 32);
             RowPartial p = warp_reduce(acc);
+            // the consumer moves on to its next item while the re-read is in flight
+            const uint32_t done = C.item;
+            acc.reset();
+            __syncwarp();
+            const uint32_t nx = item_ring[warp][consumed % ITEM_RING];
+            ++consumed;
+            open_item(job, C, nx);
             int32_t arg = INT32_MAX;
             if (holder) {
 #pragma unroll
@@ -351,13 +444,8 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
             arg = warp_min_i32(arg);
             if (lane == 0) {
                 p.argmax = arg;
-                job.partials[C.item] = p;
+                job.partials[done] = p;
             }
-            acc.reset();
-            __syncwarp();
-            const uint32_t nx = item_ring[warp][consumed % ITEM_RING];
-            ++consumed;
-            open_item(job, C, nx);
         }
         st = (st + 1 == PIPE_STAGES) ? 0 : st + 1;
     }
@@ -384,18 +472,18 @@ template <typename T, bool REV>
 __global__ void __launch_bounds__(ROW_THREADS, 4) row_reduce_generic_kernel(const RowJob job)
 {
     const int lane = threadIdx.x & 31;
-    uint32_t item = 0;
-    if (lane == 0) item = fetch_item(job);
-    item = __shfl_sync(0xffffffffu, item, 0);
+    const uint32_t workers = gridDim.x * (ROW_THREADS / 32);
+    uint32_t item = first_item(job, blockIdx.x * (ROW_THREADS / 32) + (threadIdx.x >> 5), workers, lane);
 
     while (item < job.total_items) {
         uint32_t next = 0;
-        if (lane == 0) next = fetch_item(job);   // consumed after this item
+        if (lane == 0) next = fetch_item(job, workers);   // consumed after this item
 
-        const uint32_t row = item / (uint32_t)job.segments;
-        const int32_t seg = (int32_t)(item % (uint32_t)job.segments);
-        const int32_t v0 = (int32_t)(((int64_t)job.V * seg) / job.segments);
-        const int32_t v1 = (int32_t)(((int64_t)job.V * (seg + 1)) / job.segments);
+        uint32_t row;
+        int32_t t0, t1;
+        locate_item(job.plan, item, row, t0, t1);
+        const int32_t v0 = t0 * job.tile_logits;
+        const int32_t v1 = min(t1 * job.tile_logits, job.V);
         const T *pa = reinterpret_cast<const T *>(job.target) + (size_t)row * job.V;
         const T *pb = reinterpret_cast<const T *>(job.draft) + (size_t)row * job.V;
 
@@ -431,7 +519,8 @@ struct ScanJob {
     const RowPartial *partials;
     WsHeader *header;
     ppow_outputs out;
-    int32_t N, K, V, dtype, mode, segments;
+    WorkPlan plan;
+    int32_t N, K, V, dtype, mode;
     float s;         // log2(e)/T as used by the row reduction
     float c, eta, eps;
 };
@@ -464,17 +553,20 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
     if (active) {
         const size_t row = (size_t)n * K + lane;
         // merge this row's partials against the largest references
-        const RowPartial *pp = job.partials + row * job.segments;
+        uint32_t first_part;
+        int parts;
+        row_items(job.plan, (uint32_t)row, first_part, parts);
+        const RowPartial *pp = job.partials + first_part;
         double Ra = -INFINITY, Rb = -INFINITY;
         float mx = -INFINITY;
-        for (int i = 0; i < job.segments; ++i) {
+        for (int i = 0; i < parts; ++i) {
             Ra = fmax(Ra, (double)pp[i].rho_a);
             Rb = fmax(Rb, (double)pp[i].rho_b);
             mx = fmaxf(mx, pp[i].max_a);
         }
         double Sa = 0.0, Sb = 0.0, E = 0.0, D = 0.0, Bv = 0.0;
         int32_t arg = INT32_MAX;
-        for (int i = 0; i < job.segments; ++i) {
+        for (int i = 0; i < parts; ++i) {
             const RowPartial p = pp[i];
             const double da = (double)p.rho_a - Ra, db = (double)p.rho_b - Rb;
             const double fa = exp2(da), fb = exp2(db);
@@ -601,28 +693,80 @@ static bool params_ok(const ppow_params *p)
     if (!(p->temperature > 0.0f) || !isfinite(p->temperature)) return false;
     if (!(p->c >= 0.0f) || !isfinite(p->c)) return false;
     if (!isfinite(p->eta) || !isfinite(p->eps)) return false;
-    if ((int64_t)p->N * p->K > (int64_t)1 << 26) return false;   // rows * MAX_SEGMENTS must fit 32 bits
+    if ((int64_t)p->N * p->K > (int64_t)1 << 26) return false;   // rows << MAX_SHIFT must fit 32 bits
     return true;
 }
 
-// Work items per row; depends only on (N, K, V) so that the workspace size is a pure function of
-// the parameters.  Measured on B200: an item should be as long as the balance allows (every item
-// ends with a warp reduction), so a row is cut only (a) to keep an item at or below about 64 tiles
-// of 1024 logits, and (b) to give each resident warp about four items when there are few rows;
-// never finer than 4 tiles.
+// The work plan depends only on (N, K, V, dtype), so that the workspace size is a pure function of the
+// parameters.  Measured on B200 (per-warp timeline of the kernel): an item should be as long as the
+// balance allows, because every item ends with a warp reduction worth more than half a tile of work; but
+// the warps run at speeds that differ by +-20 % and finish their last items spread over one item's
+// duration, which on a launch of a few hundred microseconds is 10-15 % of the time.  So the items shrink
+// as the work runs out (guided self-scheduling, fixed ahead of time): a row whose distance from the last
+// row leaves R tiles of work still to hand out is cut into items of at most R / (PLAN_K * resident warps)
+// tiles, rounded down to 64, 32, 16, 8 or 4.
 constexpr int64_t WORKER_WARPS = 148 * PIPE_MIN_CTAS * PIPE_WARPS;   // resident warps of the bulk-copy kernel on a B200
-static int segments_for(const ppow_params *p)
+
+static int shift_for(int64_t tiles, int64_t item_tiles)
 {
+    int sh = 0;
+    while (sh < MAX_SHIFT && ((tiles + ((int64_t)1 << sh) - 1) >> sh) > item_tiles && ((int64_t)2 << sh) <= tiles) ++sh;
+    return sh;
+}
+
+static WorkPlan make_plan(const ppow_params *p)
+{
+    WorkPlan plan;
     const int64_t rows = (int64_t)p->N * p->K;
-    if (rows <= 0) return 1;
-    const int64_t tiles = ((int64_t)p->V + 1023) / 1024;   // per row
-    int64_t seg = (4 * WORKER_WARPS + rows - 1) / rows;
-    const int64_t by_size = (tiles + 63) / 64;
-    if (seg < by_size) seg = by_size;
-    if (seg > tiles / 4) seg = tiles / 4;
-    if (seg > MAX_SEGMENTS) seg = MAX_SEGMENTS;
-    if (seg < 1) seg = 1;
-    return (int)seg;
+    const int64_t tile_logits = (int64_t)TILE_UNITS * (p->dtype == PPOW_F32 ? 4 : 8);
+    const int64_t tiles = ((int64_t)p->V + tile_logits - 1) / tile_logits;   // per row
+    plan.tiles = (int32_t)tiles;
+    // class i holds items of at most 64 >> i tiles; it starts at the first row from which at least
+    // PLAN_K * (64 >> i) * WORKER_WARPS tiles are still to come, and ends where the next class starts
+    uint32_t item = 0;
+    int64_t row = 0;
+    for (int i = 0; i < PLAN_CLASSES; ++i) {
+        int64_t end = rows;   // first row of the next class
+        if (i + 1 < PLAN_CLASSES) {
+            const int64_t from_end = (PLAN_K * (int64_t)(64 >> i) * WORKER_WARPS + tiles - 1) / tiles;
+            end = rows > from_end ? rows - from_end : 0;
+        }
+        if (end < row) end = row;
+        plan.shift[i] = shift_for(tiles, 64 >> i);
+        plan.item_begin[i] = item;
+        plan.row_begin[i] = (int32_t)row;
+        item += (uint32_t)((end - row) << plan.shift[i]);
+        row = end;
+    }
+    plan.item_begin[PLAN_CLASSES] = item;
+    plan.row_begin[PLAN_CLASSES] = (int32_t)row;
+    return plan;
+}
+
+// CTAs of a row kernel that are resident on the whole device at once.  Looked up once per (device, kernel)
+// and remembered: the dynamic shared memory opt-in, the occupancy query and the SM count are host calls
+// of several microseconds each, as much as a small problem's whole launch.  (Launch limits of a device are
+// the only thing the library remembers between calls; concurrent first calls store the same value.)
+constexpr int CACHE_DEVICES = 64, CACHE_KERNELS = 12;
+static std::atomic<int> g_resident_ctas[CACHE_DEVICES][CACHE_KERNELS];
+
+static int resident_ctas(int dev, int kernel_index, const void *kernel, int threads, size_t dyn_smem)
+{
+    const bool cached = dev >= 0 && dev < CACHE_DEVICES;
+    if (cached) {
+        const int v = g_resident_ctas[dev][kernel_index].load(std::memory_order_relaxed);
+        if (v > 0) return v;
+    }
+    int sms = 0, per_sm = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    if (dyn_smem > 0 &&
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem) != cudaSuccess)
+        return 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, dyn_smem) != cudaSuccess || per_sm < 1)
+        return 0;
+    const int v = sms * per_sm;
+    if (cached) g_resident_ctas[dev][kernel_index].store(v, std::memory_order_relaxed);
+    return v;
 }
 
 }  // namespace ppow
@@ -632,8 +776,7 @@ using namespace ppow;
 extern "C" size_t ppow_score_workspace_bytes(const ppow_params *params)
 {
     if (!params_ok(params) || params->K > 32) return 0;
-    const size_t rows = (size_t)params->N * params->K;
-    return WS_HEADER_BYTES + rows * segments_for(params) * sizeof(RowPartial);
+    return WS_HEADER_BYTES + (size_t)make_plan(params).item_begin[PLAN_CLASSES] * sizeof(RowPartial);
 }
 
 extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
@@ -659,27 +802,26 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
     RowPartial *partials = (RowPartial *)((char *)workspace + WS_HEADER_BYTES);
     if (cudaMemsetAsync(header, 0, WS_HEADER_BYTES, stream) != cudaSuccess) return PPOW_ERR_CUDA;
 
-    const int segments = segments_for(params);
+    const WorkPlan plan = make_plan(params);
     const float s = (float)(1.4426950408889634074 / (double)params->temperature);
 
     RowJob rj;
     rj.target = target_logits; rj.draft = draft_logits; rj.valid_len = valid_len;
     rj.partials = partials; rj.header = header;
     rj.N = params->N; rj.K = params->K; rj.V = params->V;
-    rj.segments = segments;
-    rj.total_items = (uint32_t)((size_t)params->N * params->K * segments);
+    rj.plan = plan;
+    rj.total_items = plan.item_begin[PLAN_CLASSES];
     rj.s = s;
 
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-        return PPOW_ERR_CUDA;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return PPOW_ERR_CUDA;
 
     // the bulk-copy kernel needs rows of whole, 16-byte aligned units; everything else takes the scalar kernel
     const int epu = params->dtype == PPOW_F32 ? FmtF32::EPU : FmtBf16::EPU;   // 8 logits per unit for both 16-bit types
     const bool vec_ok = (params->V % epu == 0) && ((uintptr_t)draft_logits % 16 == 0) &&
-                        ((uintptr_t)target_logits % 16 == 0) && (params->V / epu >= segments);
+                        ((uintptr_t)target_logits % 16 == 0);
     rj.units_per_row = params->V / epu;
+    rj.tile_logits = TILE_UNITS * epu;
     // one warp per work item in every row kernel: a grid that fills the GPU, or fewer CTAs when there is little work.
     // The kernels that also accumulate the sum for KL(Q||P) run only when that output is asked for.
     const bool rev = out->kl_rev != nullptr || out->kl_rev_mean != nullptr;
@@ -695,8 +837,6 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
             kernel = rev ? (const void *)row_reduce_pipe_kernel<true, FmtF32> : (const void *)row_reduce_pipe_kernel<false, FmtF32>;
         threads = PIPE_WARPS * 32;
         dyn_smem = PIPE_SMEM_BYTES;
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PIPE_SMEM_BYTES) != cudaSuccess)
-            return PPOW_ERR_CUDA;
     } else if (params->dtype == PPOW_BF16) {
         kernel = rev ? (const void *)row_reduce_generic_kernel<uint16_t, true>
                      : (const void *)row_reduce_generic_kernel<uint16_t, false>;
@@ -707,20 +847,23 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
         kernel = rev ? (const void *)row_reduce_generic_kernel<float, true>
                      : (const void *)row_reduce_generic_kernel<float, false>;
     }
-    int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, dyn_smem) != cudaSuccess || per_sm < 1)
-        return PPOW_ERR_CUDA;
+    const int kernel_index = (vec_ok ? 6 : 0) + 2 * params->dtype + (rev ? 1 : 0);
+    const int resident = resident_ctas(dev, kernel_index, kernel, threads, dyn_smem);
+    if (resident < 1) return PPOW_ERR_CUDA;
     const unsigned warps_per_cta = (unsigned)threads / 32;
     const unsigned ctas_needed = (rj.total_items + warps_per_cta - 1) / warps_per_cta;
-    unsigned grid = (unsigned)(sms * per_sm);
+    unsigned grid = (unsigned)resident;
     if (grid > ctas_needed) grid = ctas_needed;
 
     if (event_reduce_begin && cudaEventRecord((cudaEvent_t)event_reduce_begin, stream) != cudaSuccess)
         return PPOW_ERR_CUDA;
     void *kargs[] = {(void *)&rj};
-    if (cudaLaunchKernel(kernel, dim3(grid), dim3((unsigned)threads), kargs, dyn_smem, stream) != cudaSuccess)
+    if (cudaLaunchKernel(kernel, dim3(grid), dim3((unsigned)threads), kargs, dyn_smem, stream) != cudaSuccess ||
+        cudaGetLastError() != cudaSuccess) {
+        // a context that was torn down and rebuilt has lost the shared-memory opt-in: look the limits up again next time
+        if (dev >= 0 && dev < CACHE_DEVICES) g_resident_ctas[dev][kernel_index].store(0, std::memory_order_relaxed);
         return PPOW_ERR_CUDA;
-    if (cudaGetLastError() != cudaSuccess) return PPOW_ERR_CUDA;
+    }
     if (event_reduce_end && cudaEventRecord((cudaEvent_t)event_reduce_end, stream) != cudaSuccess)
         return PPOW_ERR_CUDA;
 
@@ -729,7 +872,7 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
     sj.valid_len = valid_len; sj.ref_logp = ref_logp; sj.partials = partials; sj.header = header;
     sj.out = *out;
     sj.N = params->N; sj.K = params->K; sj.V = params->V; sj.dtype = params->dtype; sj.mode = params->mode;
-    sj.segments = segments; sj.s = s; sj.c = params->c; sj.eta = params->eta; sj.eps = params->eps;
+    sj.plan = plan; sj.s = s; sj.c = params->c; sj.eta = params->eta; sj.eps = params->eps;
     const unsigned scan_grid = (unsigned)(((size_t)params->N * 32 + SCAN_THREADS - 1) / SCAN_THREADS);
     window_scan_kernel<<<scan_grid, SCAN_THREADS, 0, stream>>>(sj);
     if (cudaGetLastError() != cudaSuccess) return PPOW_ERR_CUDA;

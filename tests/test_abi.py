@@ -58,6 +58,18 @@ def test_host_only_entry_points(lib):
     assert B.ppow_select_workspace_bytes(100000) >= 131072 * 8
 
 
+def test_score_workspace_grows_with_the_number_of_windows(lib):
+    # the host-buffer entry point scores chunks of different sizes out of one workspace sized for the largest:
+    # a shorter chunk must never need more
+    for K, V, dt in ((8, 32000, B.PPOW_BF16), (8, 128256, B.PPOW_BF16), (10, 151936, B.PPOW_F16), (4, 1000, B.PPOW_F32),
+                     (12, 152064, B.PPOW_F32), (1, 5000, B.PPOW_BF16), (32, 777, B.PPOW_BF16)):
+        last = 0
+        for N in list(range(1, 400)) + list(range(400, 9000, 37)):
+            need = B.ppow_score_workspace_bytes(B.make_params(N, K, V, dt, B.PPOW_GREEDY, 0.05))
+            assert need >= last and need >= 256 + 64 * N * K and need <= 256 + 64 * 32 * N * K, (N, K, V)
+            last = need
+
+
 def test_binding_refuses_cpu_tensors(lib):
     import torch
     x = torch.zeros((1, 1, 8), dtype=torch.bfloat16)

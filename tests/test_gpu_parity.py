@@ -344,6 +344,33 @@ def test_host_buffer_entry_point_matches_device_path_with_chunking():
                                      B.alloc_workspace(1024, DEV))
 
 
+def test_host_buffer_entry_point_with_a_shorter_last_chunk_at_full_vocabulary_width():
+    # 477 windows staged as 296 + 181 at V = 32000: the two chunks and the whole batch are cut into work items
+    # three different ways, and the scratch size the library asks for has to serve both chunk sizes
+    w = W.scaled(W.WORKLOADS[1], 477)
+    chunk = 296
+    x = W.generate(w, DEV)
+    dev_out = run_gpu(x, "greedy", w.c, w.temperature)
+    dev_sel = B.select_windows(dev_out["score"], w.n_keep)
+    torch.cuda.synchronize()
+    params = B.make_params(w.N, w.K, w.V, B.PPOW_BF16, B.PPOW_GREEDY, w.c, w.temperature)
+    host = {k: (None if v is None else v.cpu()) for k, v in x.items()}
+    out_host = {k: torch.zeros(v.shape, dtype=v.dtype) for k, v in dev_out.items() if not k.startswith("_")}
+    sel_host = torch.zeros((w.n_keep,), dtype=torch.int32)
+    scratch = B.alloc_workspace(B.ppow_host_scratch_bytes(params, chunk), DEV)
+    B.ppow_score_and_select_host(params, host["draft_logits"], host["target_logits"], host["draft_tokens"],
+                                 None, None, None, out_host, w.n_keep, sel_host, None, scratch)
+    torch.cuda.synchronize()
+    for k, v in out_host.items():                                    # the chunks are cut into other work items than
+        if v.dtype.is_floating_point:                                # the whole batch: floats agree to rounding
+            torch.testing.assert_close(v, dev_out[k].cpu(), rtol=1e-5, atol=1e-6, msg=k)
+        else:
+            assert torch.equal(v, dev_out[k].cpu()), k
+    want = oracle.select_windows(out_host["score"].numpy().astype(np.float64), w.n_keep)
+    np.testing.assert_array_equal(sel_host.numpy(), want)
+    assert len(set(sel_host.tolist()) ^ set(dev_sel.cpu().tolist())) <= 2
+
+
 def test_randomised_shapes_parameters_and_masks():
     """Property-style sweep: seeded random shapes (odd and even V, one position to 32, one window to dozens),
     storage types, temperatures, costs, ragged masks and logit scales; everything is compared with the oracle."""
