@@ -216,6 +216,53 @@ def ppow_score_windows_traced(params: ppow_params, draft_logits, target_logits, 
         raise PpowError(st, "ppow_score_windows")
 
 
+class ScoreCall:
+    """The arguments of ``ppow_score_windows`` marshalled once.  ``launch()`` repeats the foreign call without
+    rebuilding them, which matters when the same buffers are scored step after step and the problem is small
+    enough for argument marshalling to show.  Holds references to the tensors; nothing is computed here."""
+
+    def __init__(self, params: ppow_params, draft_logits, target_logits, draft_tokens, uniforms, valid_len, ref_logp,
+                 outputs: dict, workspace: torch.Tensor):
+        self._lib = load_library()
+        lt = LOGIT_DTYPES[params.dtype]
+        self._keep = (params, draft_logits, target_logits, draft_tokens, uniforms, valid_len, ref_logp, outputs, workspace)
+        self._out = ppow_outputs()
+        for name, _ in ppow_outputs._fields_:
+            ptr = _dev_ptr(outputs.get(name), _ALL_OUTPUTS[name], name)
+            setattr(self._out, name, ptr.value if ptr is not None else None)
+        self._args = (ctypes.byref(params),
+                      _dev_ptr(draft_logits, lt, "draft_logits"), _dev_ptr(target_logits, lt, "target_logits"),
+                      _dev_ptr(draft_tokens, torch.int32, "draft_tokens"), _dev_ptr(uniforms, torch.float32, "uniforms"),
+                      _dev_ptr(valid_len, torch.int32, "valid_len"), _dev_ptr(ref_logp, torch.float32, "ref_logp"),
+                      ctypes.byref(self._out), _dev_ptr(workspace, torch.uint8, "workspace"),
+                      workspace.numel() if workspace is not None else 0)
+
+    def launch(self, stream=None, event_reduce_begin=None, event_reduce_end=None) -> None:
+        if event_reduce_begin is None and event_reduce_end is None:
+            st = self._lib.ppow_score_windows(*self._args, _stream_ptr(stream))
+        else:
+            st = self._lib.ppow_score_windows_traced(*self._args, _stream_ptr(stream), _event_ptr(event_reduce_begin),
+                                                     _event_ptr(event_reduce_end))
+        if st != PPOW_OK:
+            raise PpowError(st, "ppow_score_windows")
+
+
+class SelectCall:
+    """The arguments of ``ppow_select_windows`` marshalled once (see ScoreCall)."""
+
+    def __init__(self, score, n_keep: int, selected, mask, workspace):
+        self._lib = load_library()
+        self._keep = (score, selected, mask, workspace)
+        self._args = (_dev_ptr(score, torch.float32, "score"), int(score.numel()) if score is not None else 0, int(n_keep),
+                      _dev_ptr(selected, torch.int32, "selected"), _dev_ptr(mask, torch.uint8, "mask"),
+                      _dev_ptr(workspace, torch.uint8, "workspace"), workspace.numel() if workspace is not None else 0)
+
+    def launch(self, stream=None) -> None:
+        st = self._lib.ppow_select_windows(*self._args, _stream_ptr(stream))
+        if st != PPOW_OK:
+            raise PpowError(st, "ppow_select_windows")
+
+
 def ppow_read_error_flags(workspace: torch.Tensor, stream=None) -> int:
     lib = load_library()
     flags = ctypes.c_uint32(0)

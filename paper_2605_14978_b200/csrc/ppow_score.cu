@@ -19,6 +19,8 @@ constexpr int MAX_SHIFT = 5;       // a row is split into at most 2^5 work items
 constexpr int PLAN_CLASSES = 5;    // row classes of the work plan: items of at most 64, 32, 16, 8, 4 tiles
 constexpr int PLAN_K = 1;          // an item is at most 1/PLAN_K of a resident warp's share of the work still to hand out
 constexpr size_t WS_HEADER_BYTES = 256;
+constexpr size_t SMALL_ROW_BYTES = 4096;        // rows up to this long (at most two tiles) in
+constexpr size_t SMALL_TOTAL_BYTES = 4u << 20;  // calls up to this many logit bytes take the one-launch kernel
 
 // Workspace header (first WS_HEADER_BYTES of the workspace).
 struct WsHeader {
@@ -534,11 +536,11 @@ __device__ __forceinline__ double raw_logit(const void *base, int32_t dtype, siz
 
 constexpr int SCAN_THREADS = 128;
 
-__global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob job)
+// One warp scores window n, lane = position.  `pp` / `parts`: the partial reductions of this lane's row
+// (unused by lanes beyond the window's valid length).
+__device__ __forceinline__ void scan_window(const ScanJob &job, const int32_t n, const int lane, const RowPartial *pp,
+                                            const int parts)
 {
-    const int lane = threadIdx.x & 31;
-    const int32_t n = (int32_t)((blockIdx.x * (unsigned)SCAN_THREADS + threadIdx.x) >> 5);
-    if (n >= job.N) return;
     const int32_t K = job.K;
     int32_t L = job.valid_len ? __ldg(job.valid_len + n) : K;
     L = max(0, min(L, K));
@@ -553,10 +555,6 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
     if (active) {
         const size_t row = (size_t)n * K + lane;
         // merge this row's partials against the largest references
-        uint32_t first_part;
-        int parts;
-        row_items(job.plan, (uint32_t)row, first_part, parts);
-        const RowPartial *pp = job.partials + first_part;
         double Ra = -INFINITY, Rb = -INFINITY;
         float mx = -INFINITY;
         for (int i = 0; i < parts; ++i) {
@@ -663,6 +661,55 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
         if (job.out.score) job.out.score[n] = score;
         if (job.out.kl_rev_mean) job.out.kl_rev_mean[n] = rev_mean;
     }
+}
+
+__global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob job)
+{
+    const int lane = threadIdx.x & 31;
+    const int32_t n = (int32_t)((blockIdx.x * (unsigned)SCAN_THREADS + threadIdx.x) >> 5);
+    if (n >= job.N) return;
+    uint32_t first_part = 0;
+    int parts = 0;
+    if (lane < job.K) row_items(job.plan, (uint32_t)n * (uint32_t)job.K + (uint32_t)lane, first_part, parts);
+    scan_window(job, n, lane, job.partials + first_part, parts);
+}
+
+// ---- small problems: the whole pass in one launch ---------------------------------------------------
+// When the logits of a call are a few megabytes the pass is bound by launches, not by memory: one CTA per
+// window, warp t reduces position t's row (scalar coalesced loads, the same accumulators), the partials stay
+// in shared memory and warp 0 scores the window.  No work counter, no partials in the workspace.
+template <typename T, bool REV>
+__global__ void __launch_bounds__(1024) score_small_kernel(const RowJob rj, const ScanJob sj)
+{
+    __shared__ RowPartial parts[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int32_t n = (int32_t)blockIdx.x;
+    int32_t L = rj.valid_len ? __ldg(rj.valid_len + n) : rj.K;
+    L = max(0, min(L, rj.K));
+    if (warp < L) {
+        const size_t row = (size_t)n * rj.K + warp;
+        const T *pa = reinterpret_cast<const T *>(rj.target) + row * rj.V;
+        const T *pb = reinterpret_cast<const T *>(rj.draft) + row * rj.V;
+        RowAcc<REV> acc;
+        acc.reset();
+        int32_t arg = INT32_MAX;
+        for (int32_t v = lane; v < rj.V; v += 32) {
+            const float a = load_logit<T>(pa, v), b = load_logit<T>(pb, v);
+            acc.guard(a, b, rj.s);
+            if (a > acc.max_a) { acc.max_a = a; arg = v; }   // strict: first occurrence within the lane
+            acc.add_pair(a, b, rj.s);
+            acc.flush();
+        }
+        const float my_max = acc.max_a;
+        RowPartial p = warp_reduce(acc);
+        arg = warp_min_i32(my_max == p.max_a ? arg : INT32_MAX);
+        if (lane == 0) {
+            p.argmax = arg;
+            parts[warp] = p;
+        }
+    }
+    __syncthreads();
+    if (warp == 0) scan_window(sj, n, lane, &parts[lane < rj.K ? lane : 0], 1);
 }
 
 // ---- self-test of the bounded wait ----------------------------------------------------------------
@@ -813,6 +860,38 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
     rj.total_items = plan.item_begin[PLAN_CLASSES];
     rj.s = s;
 
+    ScanJob sj;
+    sj.target = target_logits; sj.draft = draft_logits; sj.tokens = draft_tokens; sj.uniforms = uniforms;
+    sj.valid_len = valid_len; sj.ref_logp = ref_logp; sj.partials = partials; sj.header = header;
+    sj.out = *out;
+    sj.N = params->N; sj.K = params->K; sj.V = params->V; sj.dtype = params->dtype; sj.mode = params->mode;
+    sj.plan = plan; sj.s = s; sj.c = params->c; sj.eta = params->eta; sj.eps = params->eps;
+    const bool rev = out->kl_rev != nullptr || out->kl_rev_mean != nullptr;
+
+    // a few megabytes of short rows: one launch for the whole pass (the events bracket that launch)
+    if ((size_t)params->V * esize <= SMALL_ROW_BYTES &&
+        2 * (size_t)params->N * params->K * params->V * esize <= SMALL_TOTAL_BYTES) {
+        if (event_reduce_begin && cudaEventRecord((cudaEvent_t)event_reduce_begin, stream) != cudaSuccess)
+            return PPOW_ERR_CUDA;
+        rj.units_per_row = 0;
+        rj.tile_logits = 0;
+        const dim3 grid((unsigned)params->N), block((unsigned)params->K * 32u);
+        if (params->dtype == PPOW_F32) {
+            if (rev) score_small_kernel<float, true><<<grid, block, 0, stream>>>(rj, sj);
+            else score_small_kernel<float, false><<<grid, block, 0, stream>>>(rj, sj);
+        } else if (params->dtype == PPOW_F16) {
+            if (rev) score_small_kernel<half_bits, true><<<grid, block, 0, stream>>>(rj, sj);
+            else score_small_kernel<half_bits, false><<<grid, block, 0, stream>>>(rj, sj);
+        } else {
+            if (rev) score_small_kernel<uint16_t, true><<<grid, block, 0, stream>>>(rj, sj);
+            else score_small_kernel<uint16_t, false><<<grid, block, 0, stream>>>(rj, sj);
+        }
+        if (cudaGetLastError() != cudaSuccess) return PPOW_ERR_CUDA;
+        if (event_reduce_end && cudaEventRecord((cudaEvent_t)event_reduce_end, stream) != cudaSuccess)
+            return PPOW_ERR_CUDA;
+        return PPOW_OK;
+    }
+
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return PPOW_ERR_CUDA;
 
@@ -824,7 +903,6 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
     rj.tile_logits = TILE_UNITS * epu;
     // one warp per work item in every row kernel: a grid that fills the GPU, or fewer CTAs when there is little work.
     // The kernels that also accumulate the sum for KL(Q||P) run only when that output is asked for.
-    const bool rev = out->kl_rev != nullptr || out->kl_rev_mean != nullptr;
     const void *kernel;
     int threads = ROW_THREADS;
     size_t dyn_smem = 0;
@@ -867,12 +945,6 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
     if (event_reduce_end && cudaEventRecord((cudaEvent_t)event_reduce_end, stream) != cudaSuccess)
         return PPOW_ERR_CUDA;
 
-    ScanJob sj;
-    sj.target = target_logits; sj.draft = draft_logits; sj.tokens = draft_tokens; sj.uniforms = uniforms;
-    sj.valid_len = valid_len; sj.ref_logp = ref_logp; sj.partials = partials; sj.header = header;
-    sj.out = *out;
-    sj.N = params->N; sj.K = params->K; sj.V = params->V; sj.dtype = params->dtype; sj.mode = params->mode;
-    sj.plan = plan; sj.s = s; sj.c = params->c; sj.eta = params->eta; sj.eps = params->eps;
     const unsigned scan_grid = (unsigned)(((size_t)params->N * 32 + SCAN_THREADS - 1) / SCAN_THREADS);
     window_scan_kernel<<<scan_grid, SCAN_THREADS, 0, stream>>>(sj);
     if (cudaGetLastError() != cudaSuccess) return PPOW_ERR_CUDA;

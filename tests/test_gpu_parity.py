@@ -101,6 +101,16 @@ def _both_modes(x, c=0.05, temperature=1.0, eta=1.0, eps=0.5, ref_logp=None):
     (4, 5, 8 * 2333, torch.float16),    # f16, ragged tail of units
     (7, 3, 1001, torch.float16),        # f16, scalar kernel
     (1, 8, 128256, torch.float16),      # f16, rows split into segments
+    # rows of 4 KB or less in a call of a few MB take the one-launch kernel (the cases above with V <= 1001);
+    # the same kinds of shape just past that limit reach the bulk-copy and the scalar kernels
+    (5, 1, 2056, torch.bfloat16),       # bulk-copy kernel: two tiles and one unit
+    (3, 32, 2064, torch.bfloat16),      # bulk-copy kernel, largest K
+    (7, 3, 5001, torch.bfloat16),       # odd V: scalar kernel, rows not 16-byte aligned
+    (7, 3, 3001, torch.float32),
+    (7, 3, 5001, torch.float16),
+    (2, 3, 1028, torch.float32),        # f32 bulk-copy kernel: two tiles and one unit
+    (131, 4, 1000, torch.float32),      # one-launch kernel at its size limit (4 MiB of logits)
+    (132, 4, 1000, torch.float32),      # the same rows just past the limit: bulk-copy kernel, one short item per row
 ])
 def test_shapes_and_paths(N, K, V, dtype):
     x = _random_inputs(N, K, V, dtype, seed=N * 1000 + K * 10 + V % 7)
@@ -123,8 +133,9 @@ def test_ragged_lengths_including_empty_windows():
         assert float(gpu[name][:3].float().abs().sum()) == 0.0     # empty windows: all outputs 0
 
 
-def test_unaligned_base_pointer_takes_scalar_path():
-    N, K, V = 3, 2, 512
+@pytest.mark.parametrize("V", [512, 4096])                       # one-launch kernel / scalar row kernel
+def test_unaligned_base_pointer_takes_scalar_path(V):
+    N, K = 3, 2
     x = _random_inputs(N, K, V, torch.bfloat16, seed=6)
     for key in ("target_logits", "draft_logits"):
         flat = torch.empty(N * K * V + 1, dtype=torch.bfloat16, device=DEV)
