@@ -8,23 +8,33 @@ score) and the ADAW top-fraction selection.  Default workload: the Llama-3-like 
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ppow|reference] [--workload NAME]
 
-Prints one JSON line (rank 0).  With --gpus N > 1 (launched under torch.distributed.run) every rank
-scores its own N windows; the window scores are all-gathered and every rank selects over the global
-score array (weak scaling).  --impl reference times the float64 CPU oracle instead.
+Prints one JSON line (rank 0).  Besides the K timed steps the line carries, at one GPU: the same step
+timed for at least two seconds (the regime under the board's power limit), each regime with the SM
+clocks sampled inside its own timed region; a read-only streaming pass over the same logit buffers
+(the bandwidth a kernel that only reads reaches on this GPU); the float64 CPU oracle timed on a sample
+of the same buffers and the element-by-element comparison of the GPU results with it; the end-to-end
+number through the host-buffer entry point; and one entry per other workload.  With --gpus N > 1
+(launched under torch.distributed.run) every rank scores its own N windows; the window scores are
+all-gathered and every rank selects over the global score array (weak scaling).
+--impl reference times the float64 CPU oracle instead.
 """
 import argparse
+import dataclasses
 import json
+import math
 import os
 import statistics
 import subprocess
 import sys
 import tempfile
+import threading
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+import numpy as np
 import torch
 
 from paper_2605_14978_b200 import workloads as W
@@ -32,10 +42,14 @@ from paper_2605_14978_b200 import workloads as W
 METRIC = "windows/s and logit GB/s (% of B200 HBM peak) at V=128256, K=8, N=2048"
 # DRAM bytes (read + write) per window of the row-reduction kernel from the ncu capture summarised in
 # profiles/row_reduce_pipe_bf16_llama3_like.md (256-window case; traffic grows in proportion to the
-# windows processed).  Only valid for that kernel on that workload shape.
-NCU_TRAFFIC_BYTES_PER_WINDOW = {"llama3_like": 4145686.7}
+# windows processed).  Only valid for that kernel on that workload shape; None = not re-taken since the
+# kernel last changed.
+NCU_TRAFFIC_BYTES_PER_WINDOW = {"llama3_like": None}
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+RTOL, ATOL, BAND = 1e-4, 1e-6, 1e-6      # float tolerance and the band of the stochastic acceptance test
+SUSTAINED_SECONDS = 2.0
+PARITY_SAMPLE_WINDOWS = 64               # per entry of "workloads"
 
 
 def parse_args():
@@ -51,10 +65,14 @@ def parse_args():
                     help="override the storage type of the logits (same recipe, rounded once to that type)")
     ap.add_argument("--train", action="store_true",
                     help="the step also produces the training-side quantities: KL(Q||P), nabla and the softmax "
-                         "normalisers from the scoring pass, the group-relative advantage (groups of 8), and the "
-                         "expected-acceptance pass (a second read of both logit tensors)")
+                         "normalisers from the scoring pass, the group-relative advantage (groups of 8), the "
+                         "expected-acceptance pass (a second read of both logit tensors) and the reference-window "
+                         "log-probability pass")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
-    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing and parity leg")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the >= 2 s regime")
+    ap.add_argument("--no-workloads", action="store_true", help="skip the entries for the other workloads")
+    ap.add_argument("--no-probe", action="store_true", help="skip the read-only streaming reference")
     return ap.parse_args()
 
 
@@ -67,57 +85,137 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+def config_of(w, mode):
+    """The workload description; identical in both arms for the same command line."""
+    nominal = 2 * w.N * w.K * w.V * (4 if w.dtype == "f32" else 2)
+    return {"workload": w.name, "N": w.N, "K": w.K, "V": w.V, "logits": w.dtype, "mode": mode,
+            "temperature": w.temperature, "c": w.c, "n_keep": w.n_keep,
+            "l2": ("inputs (%.2f GB per GPU) larger than L2; no flush needed" % (nominal / 1e9)) if nominal > 4e8
+            else "inputs fit L2: not an HBM figure"}
 
-    def __init__(self, index):
-        self.index = index
-        self.proc = None
-        self.file = None
+
+# ------------------------------------------------------------------------------------ clock sampling
+
+
+class ClockSampler:
+    """Samples SM clock, power and clock-event reasons (read-only NVML queries) every few milliseconds on a
+    thread, with host timestamps, so that each timed region can be given the samples that fall inside it.
+    Falls back to an `nvidia-smi -lms` child (samples of the whole run) when NVML cannot be loaded."""
+    REASONS = ((0x4, "sw_power_cap"), (0x8, "hw_slowdown"), (0x20, "sw_thermal_slowdown"),
+               (0x40, "hw_thermal_slowdown"), (0x80, "hw_power_brake_slowdown"))
+    SMI_FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+                  "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+                  "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device):
+        self.samples = []          # (t, sm_mhz, power_w, reason bits)
+        self.max_mhz = None
+        self.source = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._smi = None
+        self._handle = None
+        self._nv = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device).uuid)
+            try:
+                self._handle = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid) if not uuid.startswith("GPU-") else uuid)
+            except Exception:
+                self._handle = pynvml.nvmlDeviceGetHandleByIndex(device.index or 0)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self._handle, pynvml.NVML_CLOCK_SM))
+            self._nv = pynvml
+            self.source = "nvml"
+        except Exception:
+            self._index = device.index or 0
+            self.source = "nvidia-smi"
+
+    def _reasons(self):
+        nv = self._nv
+        for name in ("nvmlDeviceGetCurrentClocksEventReasons", "nvmlDeviceGetCurrentClocksThrottleReasons"):
+            fn = getattr(nv, name, None)
+            if fn is not None:
+                try:
+                    return int(fn(self._handle))
+                except Exception:
+                    continue
+        return 0
+
+    def _loop(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                sm = float(nv.nvmlDeviceGetClockInfo(self._handle, nv.NVML_CLOCK_SM))
+                pw = nv.nvmlDeviceGetPowerUsage(self._handle) / 1000.0
+                self.samples.append((time.perf_counter(), sm, pw, self._reasons()))
+            except Exception:
+                pass
+            self._stop.wait(0.002)
 
     def start(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+            return
         try:
-            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=self.file, stderr=subprocess.DEVNULL)
+            self._file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self._smi = subprocess.Popen(["nvidia-smi", "-i", str(self._index), "--query-gpu=" + self.SMI_FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=self._file, stderr=subprocess.DEVNULL)
         except Exception:
-            self.proc = None
+            self._smi = None
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.proc is None:
-            return out
-        time.sleep(0.15)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        self.file.flush()
-        self.file.seek(0)
-        sm, mx, reasons = [], [], set()
-        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for line in self.file:
-            parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 7:
-                continue
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+        if self._smi is not None:
+            self._smi.terminate()
             try:
-                sm.append(float(parts[0]))
-                mx.append(float(parts[1]))
-            except ValueError:
-                continue
-            for name, val in zip(names, parts[3:7]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        self.file.close()
-        os.unlink(self.file.name)
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+                self._smi.wait(timeout=5)
+            except Exception:
+                self._smi.kill()
+            self._file.flush()
+            self._file.seek(0)
+            now = time.perf_counter()
+            for line in self._file:
+                parts = [p.strip() for p in line.split(",")]
+                try:
+                    sm, mx, pw = float(parts[0]), float(parts[1]), float(parts[2])
+                except (ValueError, IndexError):
+                    continue
+                bits = 0
+                for bit, val in zip((0x8, 0x40, 0x20, 0x4), parts[3:7]):
+                    if val.lower().startswith("active"):
+                        bits |= bit
+                self.max_mhz = mx
+                self.samples.append((now, sm, pw, bits))   # no usable timestamps: whole-run samples
+            self._file.close()
+            os.unlink(self._file.name)
+
+    def region(self, t0, t1):
+        """Summary of the samples taken inside [t0, t1] (host clock)."""
+        inside = [s for s in self.samples if t0 <= s[0] <= t1] if self.source == "nvml" else list(self.samples)
+        note = None
+        if not inside and self.samples:    # a region shorter than the sampling period: the nearest sample
+            mid = 0.5 * (t0 + t1)
+            inside = [min(self.samples, key=lambda s: abs(s[0] - mid))]
+            note = "region shorter than the sampling period: nearest sample"
+        out = {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0, "source": self.source}
+        if inside:
+            bits = 0
+            for s in inside:
+                bits |= s[3]
+            out.update(sm_mhz=statistics.median(s[1] for s in inside), sm_mhz_min=min(s[1] for s in inside),
+                       power_w_max=max(s[2] for s in inside), samples=len(inside) if note is None else 0,
+                       reasons=[name for bit, name in self.REASONS if bits & bit])
+        if note:
+            out["note"] = note
         return out
+
+
+# ------------------------------------------------------------------------------------ distributed helpers
 
 
 def dist_setup(n_gpus):
@@ -149,19 +247,23 @@ def max_over_ranks(value, world, device):
     return float(t.item())
 
 
+# ------------------------------------------------------------------------------------ oracle legs
+
+
 def oracle_modes():
     import oracle
     return {"greedy": oracle.GREEDY, "stochastic": oracle.STOCHASTIC}
 
 
-def time_oracle(w, mode, x_host, n_threads):
+def run_oracle(w, mode, x_host, n_threads, n_keep):
+    """The oracle as it stands on host copies of the inputs: (seconds, outputs, selected)."""
     import oracle
     t0 = time.perf_counter()
     o = oracle.score_windows(x_host["draft_logits"], x_host["target_logits"], x_host["draft_tokens"],
                              mode=oracle_modes()[mode], c=w.c, temperature=w.temperature,
                              uniforms=x_host["uniforms"], valid_len=x_host["valid_len"], n_threads=n_threads)
-    oracle.select_windows(o["score"], min(w.n_keep, len(o["score"])))
-    return time.perf_counter() - t0
+    sel = oracle.select_windows(o["score"], min(n_keep, len(o["score"])))
+    return time.perf_counter() - t0, o, sel
 
 
 def host_sample(w, chunks, device):
@@ -169,26 +271,93 @@ def host_sample(w, chunks, device):
     return {k: (None if v is None else v.cpu()) for k, v in x.items()}
 
 
+def _outside(g, o):
+    g = np.asarray(g, np.float64)
+    o = np.asarray(o, np.float64)
+    same_inf = np.isinf(g) & np.isinf(o) & (np.sign(g) == np.sign(o))
+    with np.errstate(invalid="ignore"):
+        ok = np.abs(g - o) <= ATOL + RTOL * np.abs(o)
+    return ~(ok | same_inf)
+
+
+def parity_counts(B, w, mode, x, out, ref, ref_sel, windows, keep_pct):
+    """Counts of disagreements between the GPU outputs of the timed buffers and the oracle's outputs for the
+    windows `windows` (a slice).  Integer results must agree exactly; stochastic flags may differ only inside
+    the 1e-6 band around u = alpha (counted, and their windows left out of the accepted-length comparison);
+    floats within 1e-6 + 1e-4 |oracle|; the selection is checked on the sample's own scores."""
+    import oracle
+    fields = ("target_argmax", "accept_flag", "accepted_len", "kl", "conf", "crit", "logp_tok", "logq_tok",
+              "reward_speedup", "reward_dist", "reward", "delta", "score")
+    g = {k: out[k][windows].detach().cpu().numpy() for k in fields}
+    ints = int((g["target_argmax"] != ref["target_argmax"]).sum())
+    differ = g["accept_flag"] != ref["accept_flag"]
+    band = 0
+    band_windows = np.zeros(differ.shape[0], bool)
+    if mode == "greedy":
+        ints += int(differ.sum())
+    else:
+        u = x["uniforms"][windows].detach().cpu().numpy().astype(np.float64)
+        in_band = np.abs(ref["alpha"] - u) < BAND
+        ints += int((differ & ~in_band).sum())
+        band = int((differ & in_band).sum())
+        band_windows = differ.any(axis=1)
+    keep = ~band_windows
+    ints += int((g["accepted_len"][keep] != ref["accepted_len"][keep]).sum())
+    floats = 0
+    for f in ("kl", "conf", "crit", "logp_tok", "logq_tok"):
+        floats += int(_outside(g[f], ref[f]).sum())
+    for f in ("reward_speedup", "delta", "score"):
+        floats += int(_outside(g[f][keep], ref[f][keep]).sum())
+    near_eps = np.abs(ref["delta"] - 0.5) <= ATOL + RTOL * 0.5        # reward_dist is a threshold on delta (eps = 0.5)
+    k2 = keep & ~near_eps
+    ints += int((g["reward_dist"][k2] != ref["reward_dist"][k2].astype(np.float32)).sum())
+    floats += int(_outside(g["reward"][k2], ref["reward"][k2]).sum())
+    # selection: (i) the library's selection against the oracle's on the identical float32 scores, bit-exact;
+    # (ii) against the oracle's selection on its own float64 scores: only windows at the cut may differ
+    ns = g["score"].shape[0]
+    nk = (keep_pct * ns + 99) // 100
+    sel = B.select_windows(out["score"][windows].contiguous(), nk)
+    torch.cuda.synchronize()
+    sel = sel.cpu().numpy()
+    want = oracle.select_windows(g["score"].astype(np.float64), nk)
+    ints += int((sel != want).sum())
+    swaps = 0
+    ref_sel = oracle.select_windows(ref["score"], nk)
+    if 0 < nk < ns:
+        cut = ref["score"][ref_sel[-1]]
+        for i in set(sel.tolist()) ^ set(ref_sel.tolist()):
+            if abs(ref["score"][i] - cut) <= 2 * (ATOL + RTOL * abs(cut)):
+                swaps += 1
+            else:
+                ints += 1
+    return {"windows_checked": int(ns), "int_mismatches": ints, "float_out_of_tol": floats, "band_flags": band,
+            "near_cut_swaps": swaps}
+
+
 # -------------------------------------------------------------------------------------- reference arm
 
 
 def run_reference(args):
     """Times the float64 CPU oracle (as it stands) on the machine's host cores; rank 0 only."""
-    world, rank, local = int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")), 0
+    rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     import oracle
     oracle.build()
     w = W.BY_NAME[args.workload]
+    if args.windows:
+        w = W.scaled(w, args.windows, name=w.name)
+    if args.logits:
+        w = dataclasses.replace(w, dtype=args.logits)
     mode = args.mode or w.modes[-1]
     cores = os.cpu_count() or 1
     gen_dev = torch.device("cuda:0") if torch.cuda.is_available() else torch.device("cpu")
     n_chunks = (w.N + W.CHUNK - 1) // W.CHUNK
-    per_step = 1                                   # one chunk of 64 windows per step
-    samples = [host_sample(w, [(i * per_step) % n_chunks], gen_dev) for i in range(min(4, n_chunks))]
+    samples = [host_sample(w, [i % n_chunks], gen_dev) for i in range(min(4, n_chunks))]
     times = []
     for i in range(args.warmup + args.steps):
-        dt = time_oracle(w, mode, samples[i % len(samples)], cores)
+        xs = samples[i % len(samples)]
+        dt, _, _ = run_oracle(w, mode, xs, cores, (w.keep_pct * xs["draft_tokens"].shape[0] + 99) // 100)
         if i >= args.warmup:
             times.append(dt)
     windows = samples[0]["draft_tokens"].shape[0]
@@ -198,11 +367,10 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "windows/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "N": w.N, "K": w.K, "V": w.V, "logits": w.dtype, "mode": mode,
-                   "temperature": w.temperature, "c": w.c, "n_keep": w.n_keep},
+        "config": config_of(w, mode),
         "cpu_baseline": {"value": value, "unit": "windows/s", "cores": cores, "kind": "oracle",
-                         "sample": "%d windows of %s per step (one 64-window chunk), float64 C oracle with "
-                                   "pthreads" % (windows, w.name)},
+                         "sample": "sampled: each step scores one %d-window chunk of %s (not all N windows), float64 C "
+                                   "oracle with pthreads" % (windows, w.name)},
         "e2e": {"value": value, "unit": "windows/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -210,6 +378,157 @@ def run_reference(args):
 
 
 # -------------------------------------------------------------------------------------- ppow arm
+
+
+class Run:
+    """One workload resident on the device, with the calls of a step prepared."""
+
+    def __init__(self, B, S, w, mode, dev, rank=0, world=1, train=False):
+        self.B, self.S, self.w, self.mode, self.dev, self.world, self.train = B, S, w, mode, dev, world, train
+        n_chunks = (w.N + W.CHUNK - 1) // W.CHUNK
+        # weak scaling: rank r scores windows [r*N, (r+1)*N) of a world*N-window instance of the workload
+        wg = W.scaled(w, w.N * world, name=w.name)
+        self.x = x = W.generate(wg, dev, chunks=range(rank * n_chunks, (rank + 1) * n_chunks))
+        N, K, V = w.N, w.K, w.V
+        self.n_total, self.n_keep = N * world, wg.n_keep
+        bmode = B.PPOW_GREEDY if mode == "greedy" else B.PPOW_STOCHASTIC
+        self.params = B.make_params(N, K, V, {"f32": B.PPOW_F32, "bf16": B.PPOW_BF16, "f16": B.PPOW_F16}[w.dtype],
+                                    bmode, w.c, w.temperature)
+        self.out = B.alloc_outputs(N, K, dev)
+        if train:
+            self.out.update(B.alloc_train_outputs(N, K, dev))
+            self.advantage = torch.empty((N,), dtype=torch.float32, device=dev)
+            self.exp_accept = torch.empty((N, K), dtype=torch.float32, device=dev)
+            self.ref_logp = torch.empty((N,), dtype=torch.float32, device=dev)
+            self.row_logp = torch.empty((N, K), dtype=torch.float32, device=dev)
+            self.group = 8 if N % 8 == 0 else 1
+        self.ws = B.alloc_workspace(B.ppow_score_workspace_bytes(self.params), dev)
+        self.selected = torch.empty((self.n_keep,), dtype=torch.int32, device=dev)
+        self.sel_ws = B.alloc_workspace(B.ppow_select_workspace_bytes(self.n_total), dev)
+        self.stream = torch.cuda.current_stream()
+        self.score_call = B.ScoreCall(self.params, x["draft_logits"], x["target_logits"], x["draft_tokens"],
+                                      x["uniforms"], x["valid_len"], None, self.out, self.ws)
+        self.dtype_code = self.params.dtype
+        self.select_call = B.SelectCall(self.out["score"], self.n_keep, self.selected, None, self.sel_ws) if world == 1 else None
+        self.acc_events, self.ref_events = [], []
+        self.valid_rows = int(x["valid_len"].sum().item()) if x["valid_len"] is not None else N * K
+        self.esize = 4 if w.dtype == "f32" else 2
+        self.algo_bytes = 2 * self.valid_rows * V * self.esize    # both logit tensors, read once per launch of the row kernel
+        self.launches_per_step = B.ppow_score_kernel_launches(self.params) + 1 + (4 if train else 0)
+
+    def set_mode(self, mode):
+        """Score the same buffers under the other acceptance test."""
+        B, w, x = self.B, self.w, self.x
+        self.mode = mode
+        self.params = B.make_params(w.N, w.K, w.V, self.dtype_code, B.PPOW_GREEDY if mode == "greedy" else B.PPOW_STOCHASTIC,
+                                    w.c, w.temperature)
+        self.score_call = B.ScoreCall(self.params, x["draft_logits"], x["target_logits"], x["draft_tokens"],
+                                      x["uniforms"], x["valid_len"], None, self.out, self.ws)
+
+    def step(self, ev0=None, ev1=None):
+        B, x, out, stream = self.B, self.x, self.out, self.stream
+        self.score_call.launch(stream, ev0, ev1)
+        if self.train:
+            B.ppow_group_advantage(out["reward"], self.group, 1e-6, self.advantage, stream)
+            ea = eb = None
+            if ev0 is not None:
+                ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                ea.record(stream)
+            B.ppow_expected_acceptance(self.params, x["draft_logits"], x["target_logits"], x["valid_len"], out["lse_p"],
+                                       out["lse_q"], self.exp_accept, stream)
+            if ea is not None:
+                eb.record(stream)
+                self.acc_events.append((ea, eb))
+            # the target's logits stand in for the logits along its reference window (same shape and type)
+            B.ppow_reference_logprob(self.params, x["target_logits"], x["valid_len"], self.row_logp, self.ref_logp, stream)
+            if ea is not None:
+                ec = torch.cuda.Event(enable_timing=True)
+                ec.record(stream)
+                self.ref_events.append((eb, ec))
+        if self.world > 1:
+            scores = self.S.gather_scores(out["score"], self.n_total)    # the one exchange step
+            B.ppow_select_windows(scores, self.n_keep, self.selected, None, self.sel_ws, stream)
+        else:
+            self.select_call.launch(stream)
+
+    def measure(self, steps, warmup, trace=True):
+        """`steps` timed steps after `warmup` untimed ones.  Returns device times and the host timestamps that
+        bracket the timed region (for the clock samples).  `trace`: also time the row kernel of every step alone
+        (two more event records per step, which shows on steps of a few microseconds)."""
+        for _ in range(warmup):
+            self.step()
+        torch.cuda.synchronize()
+        ev_pairs = [((torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) if trace else (None, None))
+                    for _ in range(steps)]
+        for a, b in ev_pairs:
+            if trace:
+                a.record(), b.record()                  # create the CUDA events before the timed region
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier(self.world)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        start.record()
+        for a, b in ev_pairs:
+            self.step(a, b)
+        stop.record()
+        torch.cuda.synchronize()
+        t1 = time.perf_counter()
+        barrier(self.world)
+        elapsed_ms = max_over_ranks(start.elapsed_time(stop), self.world, self.dev)
+        reduce_ms = [a.elapsed_time(b) for a, b in ev_pairs] if trace else [float("nan")]
+        reduce_avg_ms = max_over_ranks(sum(reduce_ms) / len(reduce_ms), self.world, self.dev)
+        return {"elapsed_ms": elapsed_ms, "step_ms": elapsed_ms / steps, "kernel_ms": reduce_avg_ms, "t0": t0, "t1": t1,
+                "steps": steps}
+
+    def free(self):
+        for name in ("x", "out", "ws", "score_call", "select_call", "sel_ws", "selected"):
+            setattr(self, name, None)
+        torch.cuda.empty_cache()
+
+
+def read_only_probe(B, run, iters=10):
+    """GB/s of a read-only streaming pass (16-byte loads, XOR fold) over the run's two logit tensors."""
+    chk = torch.zeros((1,), dtype=torch.int32, device=run.dev)
+    a, b = run.x["target_logits"], run.x["draft_logits"]
+    nbytes = (a.numel() + b.numel()) * a.element_size()
+    for _ in range(2):
+        B.ppow_stream_read_probe(a, chk), B.ppow_stream_read_probe(b, chk)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(iters):
+        B.ppow_stream_read_probe(a, chk), B.ppow_stream_read_probe(b, chk)
+    e1.record()
+    torch.cuda.synchronize()
+    return nbytes * iters / (e0.elapsed_time(e1) * 1e-3) / 1e9, nbytes
+
+
+def oracle_leg(B, run, n_windows, cores):
+    """Oracle on the first n_windows of the run's buffers: timing (cpu_baseline) and parity counts."""
+    w, x = run.w, run.x
+    idx = slice(0, min(w.N, n_windows))
+    xs = {k: (None if v is None else v[idx].cpu()) for k, v in x.items()}
+    nw = xs["draft_tokens"].shape[0]
+    dt, ref, ref_sel = run_oracle(w, run.mode, xs, cores, (w.keep_pct * nw + 99) // 100)
+    parity = parity_counts(B, w, run.mode, x, run.out, ref, ref_sel, idx, w.keep_pct)
+    return dt, nw, parity
+
+
+def workload_entry(B, run, steps, sampler, peak, cores):
+    """One entry of "workloads": throughput of the row kernel and of the step, clocks inside the timed region,
+    and the parity counts of a small sample against the oracle."""
+    w, mode = run.w, run.mode
+    m = run.measure(steps, 3, trace=False)                       # the step as a caller runs it
+    m["kernel_ms"] = run.measure(min(steps, 100), 0)["kernel_ms"]    # and the row kernel alone
+    flags = B.ppow_read_error_flags(run.ws)
+    entry = {"workload": w.name, "mode": mode, "N": w.N, "K": w.K, "V": w.V, "logits": w.dtype, "steps": steps,
+             "ms_per_step": m["step_ms"], "windows_per_s": w.N / (m["step_ms"] * 1e-3),
+             "kernel_ms": m["kernel_ms"], "valid_row_bytes": run.algo_bytes,
+             "logit_gbs": run.algo_bytes / (m["kernel_ms"] * 1e-3) / 1e9,
+             "frac": run.algo_bytes / (m["kernel_ms"] * 1e-3) / 1e9 / peak,
+             "hbm_figure": run.algo_bytes > 4e8, "clocks": sampler.region(m["t0"], m["t1"]), "error_flags": flags}
+    _, _, entry["parity"] = oracle_leg(B, run, PARITY_SAMPLE_WINDOWS, cores)
+    return entry
 
 
 def run_ppow(args):
@@ -231,99 +550,76 @@ def run_ppow(args):
     if args.windows:
         w = W.scaled(w, args.windows, name=w.name)
     if args.logits:
-        import dataclasses
         w = dataclasses.replace(w, dtype=args.logits)
     mode = args.mode or w.modes[-1]
-    bmode = B.PPOW_GREEDY if mode == "greedy" else B.PPOW_STOCHASTIC
-    n_chunks = (w.N + W.CHUNK - 1) // W.CHUNK
-    # weak scaling: rank r scores windows [r*N, (r+1)*N) of a world*N-window instance of the workload
-    wg = W.scaled(w, w.N * world, name=w.name)
-    x = W.generate(wg, dev, chunks=range(rank * n_chunks, (rank + 1) * n_chunks))
+    solo = world == 1
+    cores = os.cpu_count() or 1
+    peak, peak_kind = measured_peak()
+
+    run = Run(B, S, w, mode, dev, rank, world, train=args.train)
     N, K, V = w.N, w.K, w.V
-    n_total, n_keep = N * world, wg.n_keep
-
-    params = B.make_params(N, K, V, {"f32": B.PPOW_F32, "bf16": B.PPOW_BF16, "f16": B.PPOW_F16}[w.dtype], bmode, w.c, w.temperature)
-    out = B.alloc_outputs(N, K, dev)
-    if args.train:
-        out.update(B.alloc_train_outputs(N, K, dev))
-        advantage = torch.empty((N,), dtype=torch.float32, device=dev)
-        exp_accept = torch.empty((N, K), dtype=torch.float32, device=dev)
-        ref_logp = torch.empty((N,), dtype=torch.float32, device=dev)
-        row_logp = torch.empty((N, K), dtype=torch.float32, device=dev)
-        group = 8 if N % 8 == 0 else 1
-    ws = B.alloc_workspace(B.ppow_score_workspace_bytes(params), dev)
-    selected = torch.empty((n_keep,), dtype=torch.int32, device=dev)
-    sel_ws = B.alloc_workspace(B.ppow_select_workspace_bytes(n_total), dev)
-    stream = torch.cuda.current_stream()
-
-    acc_events, ref_events = [], []
-
-    def step(ev0=None, ev1=None):
-        B.ppow_score_windows_traced(params, x["draft_logits"], x["target_logits"], x["draft_tokens"], x["uniforms"],
-                                    x["valid_len"], None, out, ws, stream, ev0, ev1)
-        if args.train:
-            B.ppow_group_advantage(out["reward"], group, 1e-6, advantage, stream)
-            ea, eb = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) if ev0 is not None else (None, None)
-            if ea is not None:
-                ea.record(stream)
-            B.ppow_expected_acceptance(params, x["draft_logits"], x["target_logits"], x["valid_len"], out["lse_p"],
-                                       out["lse_q"], exp_accept, stream)
-            if ea is not None:
-                eb.record(stream)
-                acc_events.append((ea, eb))
-            # the target's logits stand in for the logits along its reference window (same shape and type)
-            B.ppow_reference_logprob(params, x["target_logits"], x["valid_len"], row_logp, ref_logp, stream)
-            if ea is not None:
-                ec = torch.cuda.Event(enable_timing=True)
-                ec.record(stream)
-                ref_events.append((eb, ec))
-        scores = S.gather_scores(out["score"], n_total) if world > 1 else out["score"]   # the one exchange step
-        B.ppow_select_windows(scores, n_keep, selected, None, sel_ws, stream)
-
-    for _ in range(max(args.warmup, 3)):
-        step()
-    torch.cuda.synchronize()
-
-    ev_pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    for a, b in ev_pairs:
-        a.record(), b.record()                      # create the CUDA events before the timed region
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(dev.index or 0)
+    sampler = ClockSampler(dev)
     if rank == 0:
         sampler.start()
-        time.sleep(0.25)
-    barrier(world)
-    torch.cuda.synchronize()
-    start.record()
-    for a, b in ev_pairs:
-        step(a, b)
-    stop.record()
-    torch.cuda.synchronize()
-    barrier(world)
-    clocks = sampler.stop() if rank == 0 else None
-    elapsed_ms = max_over_ranks(start.elapsed_time(stop), world, dev)
-    reduce_ms = [a.elapsed_time(b) for a, b in ev_pairs]
-    reduce_avg_ms = max_over_ranks(sum(reduce_ms) / len(reduce_ms), world, dev)
-    flags = B.ppow_read_error_flags(ws)
+        time.sleep(0.05)
 
-    valid_rows = int(x["valid_len"].sum().item()) if x["valid_len"] is not None else N * K
-    esize = 4 if w.dtype == "f32" else 2
-    algo_bytes = 2 * valid_rows * V * esize         # both logit tensors, read once; per launch of the row kernel
-    peak, peak_kind = measured_peak()
-    achieved = algo_bytes / (reduce_avg_ms * 1e-3) / 1e9
+    # ---- the K timed steps (value), after W >= 3 warm-up steps
+    warmup = max(args.warmup, 3)
+    m = run.measure(args.steps, warmup)
+    flags = B.ppow_read_error_flags(run.ws)
+    clocks = sampler.region(m["t0"], m["t1"]) if rank == 0 else None
+    achieved = run.algo_bytes / (m["kernel_ms"] * 1e-3) / 1e9
+    training = None
+    if args.train:
+        acc_ms = sum(a.elapsed_time(b) for a, b in run.acc_events) / len(run.acc_events)
+        ref_ms = sum(a.elapsed_time(b) for a, b in run.ref_events) / len(run.ref_events)
+        training = {"kl_rev_in_scoring_pass": True, "group_size": run.group,
+                    "expected_acceptance_ms": acc_ms, "expected_acceptance_gbs": run.algo_bytes / (acc_ms * 1e-3) / 1e9,
+                    "reference_logprob_ms": ref_ms, "reference_logprob_gbs": 0.5 * run.algo_bytes / (ref_ms * 1e-3) / 1e9}
+
+    # ---- the same step for at least SUSTAINED_SECONDS: the regime under the board's power limit
+    sustained = None
+    if solo and not args.no_sustained and not args.train:
+        n_long = max(args.steps, int(math.ceil(SUSTAINED_SECONDS / (m["step_ms"] * 1e-3))))
+        ms = run.measure(n_long, 0)
+        cs = sampler.region(ms["t0"], ms["t1"])
+        got = run.algo_bytes / (ms["kernel_ms"] * 1e-3) / 1e9
+        sustained = {"seconds": ms["elapsed_ms"] * 1e-3, "steps": n_long, "ms_per_step": ms["step_ms"],
+                     "windows_per_s": N / (ms["step_ms"] * 1e-3), "kernel_ms": ms["kernel_ms"], "achieved": got,
+                     "frac": got / peak, "clocks": cs,
+                     "kernel_ms_x_sm_mhz": (ms["kernel_ms"] * cs["sm_mhz"]) if cs.get("sm_mhz") else None}
+
+    # ---- a read-only streaming pass over the same buffers, from the library
+    read_only = None
+    if solo and not args.no_probe:
+        gbs, nbytes = read_only_probe(B, run)
+        read_only = {"gbs": gbs, "bytes_per_pass": nbytes, "frac_of_read_only": achieved / gbs,
+                     "how": "ppow_stream_read_probe over the two logit tensors of this run, 10 passes, CUDA events"}
+
+    # ---- the oracle, as it stands, on this machine's host cores, and its outputs against the GPU's (rank 0, N = 1 only)
+    cpu_baseline = parity = None
+    if rank == 0 and solo and not args.no_cpu_baseline and not args.train:
+        import oracle
+        oracle.build()
+        n_sample = min(N, 16 * W.CHUNK)         # ~25 core-seconds of oracle work on the headline workload
+        dt, nw, parity = oracle_leg(B, run, n_sample, cores)
+        cpu_baseline = {"value": nw / dt, "unit": "windows/s", "cores": cores, "kind": "oracle",
+                        "sample": "sampled: first %d of %d windows of %s, float64 C oracle with pthreads, %.1f s wall"
+                                  % (nw, N, w.name, dt)}
 
     # ---- end to end through the host-buffer entry point: pinned host inputs -> results on the host
     e2e = None
     if not args.no_e2e:
+        x, out = run.x, run.out
         host = {k: (None if v is None else v.cpu().pin_memory()) for k, v in x.items()}
         out_host = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in out.items()}
         sel_host = torch.empty((w.n_keep,), dtype=torch.int32).pin_memory()
-        scratch = B.alloc_workspace(B.ppow_host_scratch_bytes(params, N), dev)
+        scratch = B.alloc_workspace(B.ppow_host_scratch_bytes(run.params, N), dev)
 
         def e2e_step():
-            B.ppow_score_and_select_host(params, host["draft_logits"], host["target_logits"], host["draft_tokens"],
+            B.ppow_score_and_select_host(run.params, host["draft_logits"], host["target_logits"], host["draft_tokens"],
                                          host["uniforms"], host["valid_len"], None, out_host, w.n_keep, sel_host,
-                                         None, scratch, stream)
+                                         None, scratch, run.stream)
             torch.cuda.synchronize()
             return int(sel_host[0])                 # the step's result is read on the host
 
@@ -336,56 +632,56 @@ def run_ppow(args):
         e2e_s = max_over_ranks(time.perf_counter() - t0, world, dev)
         h2d = sum(v.numel() * v.element_size() for v in host.values() if v is not None)
         d2h = sum(v.numel() * v.element_size() for v in out_host.values()) + sel_host.numel() * 4
-        e2e = {"value": n_total * e2e_steps / e2e_s, "unit": "windows/s", "h2d_bytes_per_step": h2d,
+        e2e = {"value": run.n_total * e2e_steps / e2e_s, "unit": "windows/s", "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": 1e3 * e2e_s / e2e_steps,
                "note": "ppow_score_and_select_host: pinned host logits copied to the device inside the timed region"}
-        del host, scratch
+        del host, out_host, scratch
 
-    # ---- the oracle, as it stands, on this machine's host cores (rank 0, N = 1 only)
-    cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        import oracle
-        oracle.build()
-        cores = os.cpu_count() or 1
-        n_sample_chunks = min(n_chunks, 16)     # ~25 core-seconds of oracle work on the headline workload
-        idx = slice(0, min(N, n_sample_chunks * W.CHUNK))
-        xs = {k: (None if v is None else v[idx].cpu()) for k, v in x.items()}
-        dt = time_oracle(w, mode, xs, cores)
-        nw = xs["draft_tokens"].shape[0]
-        cpu_baseline = {"value": nw / dt, "unit": "windows/s", "cores": cores, "kind": "oracle",
-                        "sample": "first %d windows of %s, float64 C oracle with pthreads, %.1f s wall" % (nw, w.name, dt)}
+    # ---- one entry per other workload (generated, timed, checked and freed one at a time)
+    workloads = None
+    launches_per_step, algo_bytes, n_total, n_keep = run.launches_per_step, run.algo_bytes, run.n_total, run.n_keep
+    if rank == 0 and solo and not args.no_workloads and args.workload == "llama3_like" and not (args.windows or args.logits or args.train):
+        run.free()
+        workloads = []
+        plan = {"tiny": 2000, "vicuna_like": 300, "qwen_like": 40, "heavy_tail": 20}
+        for ow in W.WORKLOADS:
+            if ow.name == w.name:
+                continue
+            other = Run(B, S, ow, ow.modes[0], dev)
+            for om in ow.modes:                 # heavy_tail: the same buffers under both acceptance tests
+                other.set_mode(om)
+                workloads.append(workload_entry(B, other, plan[ow.name], sampler, peak, cores))
+            other.free()
+            del other
 
+    if rank == 0:
+        sampler.stop()
     if rank != 0:
         return
-    step_ms = elapsed_ms / args.steps
-    value = n_total / (step_ms * 1e-3)
+    value = n_total / (m["step_ms"] * 1e-3)
+    per_window = NCU_TRAFFIC_BYTES_PER_WINDOW.get(w.name)
     line = {
         "metric": METRIC, "value": value, "unit": "windows/s", "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": w.name, "N_per_gpu": N, "K": K, "V": V, "logits": w.dtype, "mode": mode,
-                   "temperature": w.temperature, "c": w.c, "n_keep": n_keep,
-                   "l2": "inputs (%.2f GB per GPU) larger than L2; no flush needed" % (algo_bytes / 1e9)
-                   if algo_bytes > 4e8 else "inputs fit L2: not an HBM figure"},
-        "logit_gbs": world * algo_bytes / (step_ms * 1e-3) / 1e9,
+        "warmup": warmup, "ms_per_step": m["step_ms"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "storage_dtype": w.dtype, "data": "synthetic",
+        "config": config_of(w, mode), "n_keep_global": n_keep,
+        "logit_gbs": world * algo_bytes / (m["step_ms"] * 1e-3) / 1e9,
         "roofline": {"bound": "hbm", "kernel": "row_reduce", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                     "traffic": (NCU_TRAFFIC_BYTES_PER_WINDOW[w.name] * N
-                                 if w.name in NCU_TRAFFIC_BYTES_PER_WINDOW and w.dtype == "bf16" and not args.train else None),
-                     "traffic_source": "ncu dram__bytes_read+write on a 256-window capture, scaled by windows",
-                     "algorithmic_bytes_per_launch": algo_bytes, "kernel_ms": reduce_avg_ms},
-        "training": ({"kl_rev_in_scoring_pass": True, "group_size": group,
-                      "expected_acceptance_ms": sum(a.elapsed_time(b) for a, b in acc_events) / len(acc_events),
-                      "expected_acceptance_gbs": algo_bytes / (sum(a.elapsed_time(b) for a, b in acc_events)
-                                                               / len(acc_events) * 1e-3) / 1e9,
-                      "reference_logprob_ms": sum(a.elapsed_time(b) for a, b in ref_events) / len(ref_events),
-                      "reference_logprob_gbs": 0.5 * algo_bytes / (sum(a.elapsed_time(b) for a, b in ref_events)
-                                                                   / len(ref_events) * 1e-3) / 1e9}
-                     if args.train else None),
-        "e2e": e2e, "cpu_baseline": cpu_baseline, "gpu_launches": (7 if args.train else 3) * args.steps, "clocks": clocks,
+                     "traffic": (per_window * N if per_window and w.dtype == "bf16" and not args.train else None),
+                     "traffic_source": "ncu dram__bytes_read+write on a 256-window capture, scaled by windows "
+                                       "(null: not re-taken since the kernel last changed)",
+                     "algorithmic_bytes_per_launch": algo_bytes, "kernel_ms": m["kernel_ms"],
+                     "read_only_peak": read_only, "sustained": sustained},
+        "parity": parity, "workloads": workloads, "training": training,
+        "e2e": e2e, "cpu_baseline": cpu_baseline, "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
         "error_flags": flags,
     }
     print(json.dumps(line))
+    bad = [p for p in ([parity] + [e["parity"] for e in (workloads or [])]) if p and (p["int_mismatches"] or p["float_out_of_tol"])]
+    if bad:
+        sys.stderr.write("parity check failed: %r\n" % bad)
+        sys.exit(3)
 
 
 def main():

@@ -300,6 +300,20 @@ ppow_status ppow_score_and_select_host(const ppow_params *params,
                                        int32_t n_keep, int32_t *selected_host, uint8_t *mask_host,
                                        void *device_scratch, size_t scratch_bytes, void *cuda_stream);
 
+/*
+ * Measurement aid (an addition of this library; the paper has no counterpart): one read-only streaming pass
+ * over `bytes` of device memory with 16-byte loads, XOR-folding every 32-bit word into *checksum.  Timed with
+ * events around the call it gives the bandwidth a kernel that only reads reaches on this GPU, the ceiling the
+ * scoring pass (which reads both logit tensors once and writes next to nothing) is compared with.
+ *   data       device, 16-byte aligned; bytes a non-zero multiple of 16
+ *   checksum   device, one uint32 (cleared on the stream, then written)
+ */
+ppow_status ppow_stream_read_probe(const void *data, size_t bytes, uint32_t *checksum, void *cuda_stream);
+
+/* Number of kernels one ppow_score_windows call with these parameters launches (1: small problems are scored
+ * in a single launch; 2: row reduction + window scan; 0 on invalid parameters).  Launch accounting only. */
+int ppow_score_kernel_launches(const ppow_params *params);
+
 /* Static, never-NULL description of a status code. */
 const char *ppow_status_string(ppow_status status);
 

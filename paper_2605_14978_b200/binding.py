@@ -27,7 +27,8 @@ EXPORTS = ("ppow_score_workspace_bytes", "ppow_score_windows", "ppow_score_windo
            "ppow_select_workspace_bytes", "ppow_select_windows", "ppow_host_scratch_bytes",
            "ppow_score_and_select_host", "ppow_noalloc_scratch_bytes", "ppow_score_windows_noalloc",
            "ppow_group_advantage", "ppow_sequence_windows", "ppow_sequence_windows_mixed", "ppow_expected_acceptance",
-           "ppow_reference_logprob", "ppow_selftest_wait_timeout", "ppow_status_string", "ppow_version")
+           "ppow_reference_logprob", "ppow_selftest_wait_timeout", "ppow_stream_read_probe", "ppow_score_kernel_launches",
+           "ppow_status_string", "ppow_version")
 
 POSITION_OUTPUTS = {"accept_flag": torch.uint8, "kl": torch.float32, "conf": torch.float32, "crit": torch.float32,
                     "logp_tok": torch.float32, "logq_tok": torch.float32, "target_argmax": torch.int32}
@@ -109,6 +110,10 @@ def load_library():
     lib.ppow_reference_logprob.argtypes = [ctypes.POINTER(ppow_params), vp, vp, vp, vp, vp]
     lib.ppow_selftest_wait_timeout.restype = ctypes.c_int
     lib.ppow_selftest_wait_timeout.argtypes = [vp, sz, ctypes.c_uint32, vp]
+    lib.ppow_stream_read_probe.restype = ctypes.c_int
+    lib.ppow_stream_read_probe.argtypes = [vp, sz, vp, vp]
+    lib.ppow_score_kernel_launches.restype = ctypes.c_int
+    lib.ppow_score_kernel_launches.argtypes = [ctypes.POINTER(ppow_params)]
     lib.ppow_status_string.restype = ctypes.c_char_p
     lib.ppow_status_string.argtypes = [ctypes.c_int]
     lib.ppow_version.restype = ctypes.c_int
@@ -150,6 +155,20 @@ def make_params(N, K, V, dtype, mode, c, temperature=1.0, eta=1.0, eps=0.5) -> p
 
 def ppow_score_workspace_bytes(params: ppow_params) -> int:
     return int(load_library().ppow_score_workspace_bytes(ctypes.byref(params)))
+
+
+def ppow_score_kernel_launches(params: ppow_params) -> int:
+    return int(load_library().ppow_score_kernel_launches(ctypes.byref(params)))
+
+
+def ppow_stream_read_probe(data: torch.Tensor, checksum: torch.Tensor, stream=None) -> None:
+    """One read-only streaming pass over ``data`` (any dtype, contiguous, a multiple of 16 bytes); XOR of its
+    32-bit words into ``checksum`` (one int32/uint32-sized CUDA element)."""
+    lib = load_library()
+    st = lib.ppow_stream_read_probe(_dev_ptr(data, None, "data"), data.numel() * data.element_size(),
+                                    _dev_ptr(checksum, None, "checksum"), _stream_ptr(stream))
+    if st != PPOW_OK:
+        raise PpowError(st, "ppow_stream_read_probe")
 
 
 def ppow_select_workspace_bytes(N: int) -> int:

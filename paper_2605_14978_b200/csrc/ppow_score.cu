@@ -790,6 +790,12 @@ static WorkPlan make_plan(const ppow_params *p)
     return plan;
 }
 
+static bool takes_small_path(const ppow_params *p)
+{
+    const size_t esize = p->dtype == PPOW_F32 ? 4 : 2;
+    return (size_t)p->V * esize <= SMALL_ROW_BYTES && 2 * (size_t)p->N * p->K * p->V * esize <= SMALL_TOTAL_BYTES;
+}
+
 // CTAs of a row kernel that are resident on the whole device at once.  Looked up once per (device, kernel)
 // and remembered: the dynamic shared memory opt-in, the occupancy query and the SM count are host calls
 // of several microseconds each, as much as a small problem's whole launch.  (Launch limits of a device are
@@ -824,6 +830,12 @@ extern "C" size_t ppow_score_workspace_bytes(const ppow_params *params)
 {
     if (!params_ok(params) || params->K > 32) return 0;
     return WS_HEADER_BYTES + (size_t)make_plan(params).item_begin[PLAN_CLASSES] * sizeof(RowPartial);
+}
+
+extern "C" int ppow_score_kernel_launches(const ppow_params *params)
+{
+    if (!params_ok(params) || params->K > 32 || params->N == 0) return 0;
+    return takes_small_path(params) ? 1 : 2;
 }
 
 extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
@@ -869,8 +881,7 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
     const bool rev = out->kl_rev != nullptr || out->kl_rev_mean != nullptr;
 
     // a few megabytes of short rows: one launch for the whole pass (the events bracket that launch)
-    if ((size_t)params->V * esize <= SMALL_ROW_BYTES &&
-        2 * (size_t)params->N * params->K * params->V * esize <= SMALL_TOTAL_BYTES) {
+    if (takes_small_path(params)) {
         if (event_reduce_begin && cudaEventRecord((cudaEvent_t)event_reduce_begin, stream) != cudaSuccess)
             return PPOW_ERR_CUDA;
         rj.units_per_row = 0;
