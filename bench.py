@@ -531,6 +531,17 @@ def workload_entry(B, run, steps, sampler, peak, cores):
     return entry
 
 
+def training_figures(run, m):
+    """Throughput of the training-side streaming kernels of a --train run (row kernel with the KL(Q||P) sum,
+    expected-acceptance pass over both tensors, reference-window log-probability pass over one)."""
+    acc_ms = sum(a.elapsed_time(b) for a, b in run.acc_events) / len(run.acc_events)
+    ref_ms = sum(a.elapsed_time(b) for a, b in run.ref_events) / len(run.ref_events)
+    return {"logits": run.w.dtype, "kl_rev_in_scoring_pass": True, "group_size": run.group,
+            "row_reduce_with_kl_rev_ms": m["kernel_ms"], "row_reduce_with_kl_rev_gbs": run.algo_bytes / (m["kernel_ms"] * 1e-3) / 1e9,
+            "expected_acceptance_ms": acc_ms, "expected_acceptance_gbs": run.algo_bytes / (acc_ms * 1e-3) / 1e9,
+            "reference_logprob_ms": ref_ms, "reference_logprob_gbs": 0.5 * run.algo_bytes / (ref_ms * 1e-3) / 1e9}
+
+
 def run_ppow(args):
     from paper_2605_14978_b200 import binding as B
     from paper_2605_14978_b200 import build as build_mod
@@ -569,13 +580,7 @@ def run_ppow(args):
     flags = B.ppow_read_error_flags(run.ws)
     clocks = sampler.region(m["t0"], m["t1"]) if rank == 0 else None
     achieved = run.algo_bytes / (m["kernel_ms"] * 1e-3) / 1e9
-    training = None
-    if args.train:
-        acc_ms = sum(a.elapsed_time(b) for a, b in run.acc_events) / len(run.acc_events)
-        ref_ms = sum(a.elapsed_time(b) for a, b in run.ref_events) / len(run.ref_events)
-        training = {"kl_rev_in_scoring_pass": True, "group_size": run.group,
-                    "expected_acceptance_ms": acc_ms, "expected_acceptance_gbs": run.algo_bytes / (acc_ms * 1e-3) / 1e9,
-                    "reference_logprob_ms": ref_ms, "reference_logprob_gbs": 0.5 * run.algo_bytes / (ref_ms * 1e-3) / 1e9}
+    training = training_figures(run, m) if args.train else None
 
     # ---- the same step for at least SUSTAINED_SECONDS: the regime under the board's power limit
     sustained = None
@@ -653,6 +658,16 @@ def run_ppow(args):
                 workloads.append(workload_entry(B, other, plan[ow.name], sampler, peak, cores))
             other.free()
             del other
+        # the training-side streaming kernels on the headline shape in each storage type
+        training = []
+        for lg in ("bf16", "f16", "f32"):
+            tr = Run(B, S, dataclasses.replace(w, dtype=lg), mode, dev, train=True)
+            mt = tr.measure(20, 3)
+            fig = training_figures(tr, mt)
+            fig["clocks"] = sampler.region(mt["t0"], mt["t1"])
+            training.append(fig)
+            tr.free()
+            del tr
 
     if rank == 0:
         sampler.stop()

@@ -178,6 +178,69 @@ struct RowAcc {
     }
 };
 
+// ---- storage formats: one 16-byte unit of logits, and one logit at a time ---------------------------
+
+struct UnitBf16 {
+    static constexpr int EPU = 8;   // logits per unit
+    static __device__ __forceinline__ uint4 none() { return make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u); }
+    static __device__ __forceinline__ float unit_max(const uint4 &w)
+    {
+        const uint32_t m = max_bf16x2(max_bf16x2(w.x, w.y), max_bf16x2(w.z, w.w));
+        return fmaxf(bf16_lo(m), bf16_hi(m));
+    }
+    static __device__ __forceinline__ void unpack(const uint4 &w, float (&f)[8])
+    {
+        f[0] = bf16_lo(w.x); f[1] = bf16_hi(w.x); f[2] = bf16_lo(w.y); f[3] = bf16_hi(w.y);
+        f[4] = bf16_lo(w.z); f[5] = bf16_hi(w.z); f[6] = bf16_lo(w.w); f[7] = bf16_hi(w.w);
+    }
+};
+
+struct UnitF16 {
+    static constexpr int EPU = 8;
+    static __device__ __forceinline__ uint4 none() { return make_uint4(0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u); }
+    static __device__ __forceinline__ __half2 h2(uint32_t w) { return *reinterpret_cast<const __half2 *>(&w); }
+    static __device__ __forceinline__ float unit_max(const uint4 &w)
+    {
+        const float2 f = __half22float2(__hmax2(__hmax2(h2(w.x), h2(w.y)), __hmax2(h2(w.z), h2(w.w))));
+        return fmaxf(f.x, f.y);
+    }
+    static __device__ __forceinline__ void unpack(const uint4 &w, float (&f)[8])
+    {
+        const float2 a = __half22float2(h2(w.x)), b = __half22float2(h2(w.y));
+        const float2 c = __half22float2(h2(w.z)), d = __half22float2(h2(w.w));
+        f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y; f[4] = c.x; f[5] = c.y; f[6] = d.x; f[7] = d.y;
+    }
+};
+
+struct UnitF32 {
+    static constexpr int EPU = 4;
+    static __device__ __forceinline__ uint4 none() { return make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u); }
+    static __device__ __forceinline__ float unit_max(const uint4 &w)
+    {
+        return fmaxf(fmaxf(__uint_as_float(w.x), __uint_as_float(w.y)), fmaxf(__uint_as_float(w.z), __uint_as_float(w.w)));
+    }
+    static __device__ __forceinline__ void unpack(const uint4 &w, float (&f)[4])
+    {
+        f[0] = __uint_as_float(w.x); f[1] = __uint_as_float(w.y); f[2] = __uint_as_float(w.z); f[3] = __uint_as_float(w.w);
+    }
+};
+
+// One stored logit widened to f32 (T: float, uint16_t = bf16 bits, half_bits = IEEE binary16 bits).
+template <typename T>
+__device__ __forceinline__ float load_logit(const T *p, size_t i);
+template <>
+__device__ __forceinline__ float load_logit<float>(const float *p, size_t i) { return __ldcs(p + i); }
+template <>
+__device__ __forceinline__ float load_logit<uint16_t>(const uint16_t *p, size_t i)
+{
+    return __uint_as_float(((uint32_t)__ldcs(p + i)) << 16);
+}
+template <>
+__device__ __forceinline__ float load_logit<half_bits>(const half_bits *p, size_t i)
+{
+    return f16_to_f32(__ldcs(&p[i].bits));
+}
+
 // Maximum over the warp in one instruction (sm_100a reduces f32 min/max in hardware).
 __device__ __forceinline__ float warp_max(float v)
 {

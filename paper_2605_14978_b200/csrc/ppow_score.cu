@@ -455,21 +455,6 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
 
 // ---- generic path: any V, any alignment, f32 or bf16 -------------------------------------------
 
-template <typename T>
-__device__ __forceinline__ float load_logit(const T *p, size_t i);
-template <>
-__device__ __forceinline__ float load_logit<float>(const float *p, size_t i) { return __ldcs(p + i); }
-template <>
-__device__ __forceinline__ float load_logit<uint16_t>(const uint16_t *p, size_t i)
-{
-    return __uint_as_float(((uint32_t)__ldcs(p + i)) << 16);
-}
-template <>
-__device__ __forceinline__ float load_logit<half_bits>(const half_bits *p, size_t i)
-{
-    return f16_to_f32(__ldcs(&p[i].bits));
-}
-
 template <typename T, bool REV>
 __global__ void __launch_bounds__(ROW_THREADS, 4) row_reduce_generic_kernel(const RowJob job)
 {

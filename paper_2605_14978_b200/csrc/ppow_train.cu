@@ -3,20 +3,11 @@
 // acceptance probability sum_v min(P, Q) (App. B.1).  The first two are tiny; the third streams both
 // logit tensors a second time.
 #include "../../include/ppow.h"
+#include "ppow_device.cuh"
 
-#include <cuda_fp16.h>
-#include <cuda_runtime.h>
 #include <math.h>
-#include <stdint.h>
 
 namespace ppow {
-
-__device__ __forceinline__ double warp_sum_double(double v)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-}
 
 // ---- group-relative advantage: one warp per rollout group ------------------------------------------
 constexpr int ADV_THREADS = 128;
@@ -31,13 +22,13 @@ __global__ void __launch_bounds__(ADV_THREADS) group_advantage_kernel(const floa
     const float *r = reward + (size_t)g * G;
     double sum = 0.0;
     for (int32_t i = lane; i < G; i += 32) sum += (double)r[i];
-    const double mu = warp_sum_double(sum) / (double)G;
+    const double mu = warp_sum_f64(sum) / (double)G;
     double sq = 0.0;
     for (int32_t i = lane; i < G; i += 32) {
         const double d = (double)r[i] - mu;
         sq += d * d;
     }
-    const double sigma = sqrt(warp_sum_double(sq) / (double)G);   // population standard deviation
+    const double sigma = sqrt(warp_sum_f64(sq) / (double)G);   // population standard deviation
     for (int32_t i = lane; i < G; i += 32)
         advantage[(size_t)g * G + i] = (float)(((double)r[i] - mu) / (sigma + delta));
 }
@@ -145,39 +136,16 @@ __global__ void __launch_bounds__(SEQ_THREADS) sequence_windows_kernel(const flo
 // ---- expected acceptance: one CTA per (window, position) row ---------------------------------------
 constexpr int ACC_THREADS = 256;
 
-__device__ __forceinline__ float ex2f(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-template <typename T>
-__device__ __forceinline__ float logit_at(const T *p, size_t i);
-template <>
-__device__ __forceinline__ float logit_at<float>(const float *p, size_t i) { return __ldcs(p + i); }
-template <>
-__device__ __forceinline__ float logit_at<uint16_t>(const uint16_t *p, size_t i)   // bf16 bit patterns
-{
-    return __uint_as_float(((uint32_t)__ldcs(p + i)) << 16);
-}
-struct half_bits {   // IEEE binary16 bit patterns
-    uint16_t bits;
-};
-template <>
-__device__ __forceinline__ float logit_at<half_bits>(const half_bits *p, size_t i)
-{
-    return __half2float(__ushort_as_half(__ldcs(&p[i].bits)));
-}
-
-// VEC: bf16 rows of whole, 16-byte aligned 8-logit units.
-template <typename T, bool VEC>
-__global__ void __launch_bounds__(ACC_THREADS) expected_acceptance_kernel(const T *__restrict__ target,
-                                                                          const T *__restrict__ draft,
-                                                                          const int32_t *__restrict__ valid_len,
-                                                                          const float *__restrict__ lse_p,
-                                                                          const float *__restrict__ lse_q, int32_t K,
-                                                                          int32_t V, float s, float *__restrict__ out)
+// Rows of whole, 16-byte aligned units of any storage format: 16-byte streaming loads, two units of each
+// tensor in flight per thread.
+template <typename Unit>
+__global__ void __launch_bounds__(ACC_THREADS) expected_acceptance_vec_kernel(const uint4 *__restrict__ target,
+                                                                              const uint4 *__restrict__ draft,
+                                                                              const int32_t *__restrict__ valid_len,
+                                                                              const float *__restrict__ lse_p,
+                                                                              const float *__restrict__ lse_q, int32_t K,
+                                                                              int32_t units, float s,
+                                                                              float *__restrict__ out)
 {
     __shared__ double warp_part[ACC_THREADS / 32];
     const size_t row = blockIdx.x;
@@ -189,29 +157,60 @@ __global__ void __launch_bounds__(ACC_THREADS) expected_acceptance_kernel(const 
     }
     // P(v) = 2^(a*s - la), Q(v) = 2^(b*s - lb) with the normalisers converted to log2 units
     const float la = lse_p[row] * 1.4426950408889634f, lb = lse_q[row] * 1.4426950408889634f;
+    const uint4 *pa = target + row * (size_t)units, *pb = draft + row * (size_t)units;
     float acc0 = 0.0f, acc1 = 0.0f;
-    if (VEC) {
-        const uint4 *pa = reinterpret_cast<const uint4 *>(target) + row * (size_t)(V >> 3);
-        const uint4 *pb = reinterpret_cast<const uint4 *>(draft) + row * (size_t)(V >> 3);
-        for (int32_t u = tid; u < (V >> 3); u += ACC_THREADS) {
-            const uint4 A = __ldcs(pa + u), B = __ldcs(pb + u);
-            const uint32_t wa[4] = {A.x, A.y, A.z, A.w}, wb[4] = {B.x, B.y, B.z, B.w};
+    auto add_unit = [&](const uint4 &A, const uint4 &B) {
+        float fa[Unit::EPU], fb[Unit::EPU];
+        Unit::unpack(A, fa);
+        Unit::unpack(B, fb);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const float p0 = ex2f(fmaf(__uint_as_float(wa[q] << 16), s, -la));
-                const float q0 = ex2f(fmaf(__uint_as_float(wb[q] << 16), s, -lb));
-                const float p1 = ex2f(fmaf(__uint_as_float(wa[q] & 0xffff0000u), s, -la));
-                const float q1 = ex2f(fmaf(__uint_as_float(wb[q] & 0xffff0000u), s, -lb));
-                acc0 += fminf(p0, q0);
-                acc1 += fminf(p1, q1);
-            }
+        for (int e = 0; e < Unit::EPU; e += 2) {
+            acc0 += fminf(ex2_approx(fmaf(fa[e], s, -la)), ex2_approx(fmaf(fb[e], s, -lb)));
+            acc1 += fminf(ex2_approx(fmaf(fa[e + 1], s, -la)), ex2_approx(fmaf(fb[e + 1], s, -lb)));
         }
-    } else {
-        const T *pa = target + row * (size_t)V, *pb = draft + row * (size_t)V;
-        for (int32_t v = tid; v < V; v += ACC_THREADS)
-            acc0 += fminf(ex2f(fmaf(logit_at<T>(pa, v), s, -la)), ex2f(fmaf(logit_at<T>(pb, v), s, -lb)));
+    };
+    int32_t u = tid;
+    for (; u + ACC_THREADS < units; u += 2 * ACC_THREADS) {
+        const uint4 A0 = __ldcs(pa + u), B0 = __ldcs(pb + u);
+        const uint4 A1 = __ldcs(pa + u + ACC_THREADS), B1 = __ldcs(pb + u + ACC_THREADS);
+        add_unit(A0, B0);
+        add_unit(A1, B1);
     }
-    const double w = warp_sum_double((double)acc0 + (double)acc1);
+    if (u < units) add_unit(__ldcs(pa + u), __ldcs(pb + u));
+    const double w = warp_sum_f64((double)acc0 + (double)acc1);
+    if ((tid & 31) == 0) warp_part[tid >> 5] = w;
+    __syncthreads();
+    if (tid == 0) {
+        double t = 0.0;
+#pragma unroll
+        for (int i = 0; i < ACC_THREADS / 32; ++i) t += warp_part[i];
+        out[row] = (float)fmin(t, 1.0);
+    }
+}
+
+// Any V, any alignment: one logit per load.
+template <typename T>
+__global__ void __launch_bounds__(ACC_THREADS) expected_acceptance_scalar_kernel(const T *__restrict__ target,
+                                                                                 const T *__restrict__ draft,
+                                                                                 const int32_t *__restrict__ valid_len,
+                                                                                 const float *__restrict__ lse_p,
+                                                                                 const float *__restrict__ lse_q, int32_t K,
+                                                                                 int32_t V, float s, float *__restrict__ out)
+{
+    __shared__ double warp_part[ACC_THREADS / 32];
+    const size_t row = blockIdx.x;
+    const int32_t n = (int32_t)(row / (size_t)K), k = (int32_t)(row % (size_t)K);
+    const int tid = threadIdx.x;
+    if (valid_len && k >= valid_len[n]) {
+        if (tid == 0) out[row] = 0.0f;
+        return;
+    }
+    const float la = lse_p[row] * 1.4426950408889634f, lb = lse_q[row] * 1.4426950408889634f;
+    const T *pa = target + row * (size_t)V, *pb = draft + row * (size_t)V;
+    float acc = 0.0f;
+    for (int32_t v = tid; v < V; v += ACC_THREADS)
+        acc += fminf(ex2_approx(fmaf(load_logit<T>(pa, v), s, -la)), ex2_approx(fmaf(load_logit<T>(pb, v), s, -lb)));
+    const double w = warp_sum_f64((double)acc);
     if ((tid & 31) == 0) warp_part[tid >> 5] = w;
     __syncthreads();
     if (tid == 0) {
@@ -227,13 +226,6 @@ __global__ void __launch_bounds__(ACC_THREADS) expected_acceptance_kernel(const 
 // group of logits exceeds it by 2^4), group-local f32 partial folded into a compensated (hi, lo) pair,
 // merged across the block in float64.  log max_v P(v) = ln2 * (M*s - R - log2 S).
 constexpr int REF_THREADS = 256;
-
-__device__ __forceinline__ uint32_t max_bf16x2_(uint32_t a, uint32_t b)
-{
-    uint32_t d;
-    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-    return d;
-}
 
 struct LseAcc {
     float rho, S, S_hi, S_lo, m;
@@ -256,70 +248,23 @@ struct LseAcc {
         m = fmaxf(m, group_max);
         if (fmaf(group_max, s, -rho) > 4.0f) {
             fold();
-            const float nr = group_max * s, f = ex2f(rho - nr);
+            const float nr = group_max * s, f = ex2_approx(rho - nr);
             S_hi *= f;
             S_lo *= f;
             rho = nr;
         }
     }
-    __device__ __forceinline__ void add(float v, float s) { S += ex2f(fmaf(v, s, -rho)); }
+    __device__ __forceinline__ void add(float v, float s) { S += ex2_approx(fmaf(v, s, -rho)); }
 };
 
-// One CTA per (window, position) row from a plain grid; writes log max_v P(v) of the row.
-template <typename T, bool VEC>
-__global__ void __launch_bounds__(REF_THREADS) reference_logprob_rows_kernel(const T *__restrict__ ref,
-                                                                             const int32_t *__restrict__ valid_len,
-                                                                             int32_t K, int32_t V, float s,
-                                                                             float *__restrict__ row_logp)
+// Block merge of the per-thread sums against the largest reference; thread 0 writes the row's value.
+__device__ __forceinline__ void lse_block_finish(const LseAcc &acc, float s, float *row_logp_out)
 {
     __shared__ float sh_rho[REF_THREADS / 32], sh_m[REF_THREADS / 32];
     __shared__ double sh_S[REF_THREADS / 32];
-    const size_t row = blockIdx.x;
-    const int32_t n = (int32_t)(row / (size_t)K), k = (int32_t)(row % (size_t)K);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (valid_len && k >= valid_len[n]) {
-        if (tid == 0) row_logp[row] = 0.0f;
-        return;
-    }
-    LseAcc acc;
-    acc.reset();
-    if (VEC) {
-        const uint4 *p = reinterpret_cast<const uint4 *>(ref) + row * (size_t)(V >> 3);
-        const int32_t units = V >> 3;
-        for (int32_t u = tid; u < units; u += 2 * REF_THREADS) {
-            const bool two = u + REF_THREADS < units;
-            const uint4 w0 = __ldcs(p + u);
-            const uint4 w1 = two ? __ldcs(p + u + REF_THREADS) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
-            uint32_t mx = max_bf16x2_(max_bf16x2_(max_bf16x2_(w0.x, w0.y), max_bf16x2_(w0.z, w0.w)),
-                                      max_bf16x2_(max_bf16x2_(w1.x, w1.y), max_bf16x2_(w1.z, w1.w)));
-            acc.guard(fmaxf(__uint_as_float(mx << 16), __uint_as_float(mx & 0xffff0000u)), s);
-            const uint32_t w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                if (q < 4 || two) {
-                    acc.add(__uint_as_float(w[q] << 16), s);
-                    acc.add(__uint_as_float(w[q] & 0xffff0000u), s);
-                }
-            }
-            acc.fold();
-        }
-    } else {
-        const T *p = ref + row * (size_t)V;
-        for (int32_t i = tid; i < V; i += REF_THREADS) {
-            const float v = logit_at<T>(p, i);
-            acc.guard(v, s);
-            acc.add(v, s);
-            acc.fold();
-        }
-    }
-    // block merge against the largest reference
-    float R = acc.rho, M = acc.m;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        R = fmaxf(R, __shfl_xor_sync(0xffffffffu, R, o));
-        M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-    }
-    const double Sw = warp_sum_double(exp2((double)acc.rho - (double)R) * ((double)acc.S_hi + (double)acc.S_lo));
+    const float R = warp_max(acc.rho), M = warp_max(acc.m);
+    const double Sw = warp_sum_f64(exp2((double)acc.rho - (double)R) * ((double)acc.S_hi + (double)acc.S_lo));
     if (lane == 0) {
         sh_rho[warp] = R;
         sh_m[warp] = M;
@@ -336,8 +281,80 @@ __global__ void __launch_bounds__(REF_THREADS) reference_logprob_rows_kernel(con
         double Sb = 0.0;
 #pragma unroll
         for (int i = 0; i < REF_THREADS / 32; ++i) Sb += exp2((double)sh_rho[i] - (double)Rb) * sh_S[i];
-        row_logp[row] = (float)((fma((double)Mb, (double)s, -(double)Rb) - log2(Sb)) * 0.69314718055994530942);
+        *row_logp_out = (float)((fma((double)Mb, (double)s, -(double)Rb) - log2(Sb)) * 0.69314718055994530942);
     }
+}
+
+// One CTA per (window, position) row from a plain grid; writes log max_v P(v) of the row.
+// Rows of whole, 16-byte aligned units of any storage format (one fold per 8 or 16 logits).
+template <typename Unit>
+__global__ void __launch_bounds__(REF_THREADS) reference_logprob_vec_kernel(const uint4 *__restrict__ ref,
+                                                                            const int32_t *__restrict__ valid_len,
+                                                                            int32_t K, int32_t units, float s,
+                                                                            float *__restrict__ row_logp)
+{
+    const size_t row = blockIdx.x;
+    const int32_t n = (int32_t)(row / (size_t)K), k = (int32_t)(row % (size_t)K);
+    const int tid = threadIdx.x;
+    if (valid_len && k >= valid_len[n]) {
+        if (tid == 0) row_logp[row] = 0.0f;
+        return;
+    }
+    LseAcc acc;
+    acc.reset();
+    const uint4 *p = ref + row * (size_t)units;
+    auto add_unit = [&](const uint4 &w) {
+        float f[Unit::EPU];
+        Unit::unpack(w, f);
+#pragma unroll
+        for (int e = 0; e < Unit::EPU; ++e) acc.add(f[e], s);
+    };
+    // four units of the row in flight per thread (a single tensor is read: fewer loads per thread would leave
+    // the memory system short of requests), one reference check and one fold per round
+    int32_t u = tid;
+    for (; u + 3 * REF_THREADS < units; u += 4 * REF_THREADS) {
+        const uint4 w0 = __ldcs(p + u), w1 = __ldcs(p + u + REF_THREADS);
+        const uint4 w2 = __ldcs(p + u + 2 * REF_THREADS), w3 = __ldcs(p + u + 3 * REF_THREADS);
+        acc.guard(fmaxf(fmaxf(Unit::unit_max(w0), Unit::unit_max(w1)), fmaxf(Unit::unit_max(w2), Unit::unit_max(w3))), s);
+        add_unit(w0);
+        add_unit(w1);
+        acc.fold();
+        add_unit(w2);
+        add_unit(w3);
+        acc.fold();
+    }
+    for (; u < units; u += REF_THREADS) {
+        const uint4 w0 = __ldcs(p + u);
+        acc.guard(Unit::unit_max(w0), s);
+        add_unit(w0);
+        acc.fold();
+    }
+    lse_block_finish(acc, s, row_logp + row);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(REF_THREADS) reference_logprob_scalar_kernel(const T *__restrict__ ref,
+                                                                               const int32_t *__restrict__ valid_len,
+                                                                               int32_t K, int32_t V, float s,
+                                                                               float *__restrict__ row_logp)
+{
+    const size_t row = blockIdx.x;
+    const int32_t n = (int32_t)(row / (size_t)K), k = (int32_t)(row % (size_t)K);
+    const int tid = threadIdx.x;
+    if (valid_len && k >= valid_len[n]) {
+        if (tid == 0) row_logp[row] = 0.0f;
+        return;
+    }
+    LseAcc acc;
+    acc.reset();
+    const T *p = ref + row * (size_t)V;
+    for (int32_t i = tid; i < V; i += REF_THREADS) {
+        const float v = load_logit<T>(p, i);
+        acc.guard(v, s);
+        acc.add(v, s);
+        acc.fold();
+    }
+    lse_block_finish(acc, s, row_logp + row);
 }
 
 // ref_logp[n] = sum of the window's row values, added in position order (float64).
@@ -416,22 +433,24 @@ extern "C" ppow_status ppow_expected_acceptance(const ppow_params *params,
     const unsigned rows = (unsigned)((size_t)params->N * params->K);
     const float s = (float)(1.4426950408889634074 / (double)params->temperature);
     const int32_t K = params->K, V = params->V;
-    if (params->dtype == PPOW_F32) {
-        expected_acceptance_kernel<float, false><<<rows, ACC_THREADS, 0, stream>>>(
+    const int epu = params->dtype == PPOW_F32 ? 4 : 8;
+    const bool vec = V % epu == 0 && (uintptr_t)draft_logits % 16 == 0 && (uintptr_t)target_logits % 16 == 0;
+    const uint4 *ta = (const uint4 *)target_logits, *da = (const uint4 *)draft_logits;
+    if (vec && params->dtype == PPOW_BF16)
+        expected_acceptance_vec_kernel<UnitBf16><<<rows, ACC_THREADS, 0, stream>>>(ta, da, valid_len, lse_p, lse_q, K, V / epu, s, expected_accept);
+    else if (vec && params->dtype == PPOW_F16)
+        expected_acceptance_vec_kernel<UnitF16><<<rows, ACC_THREADS, 0, stream>>>(ta, da, valid_len, lse_p, lse_q, K, V / epu, s, expected_accept);
+    else if (vec)
+        expected_acceptance_vec_kernel<UnitF32><<<rows, ACC_THREADS, 0, stream>>>(ta, da, valid_len, lse_p, lse_q, K, V / epu, s, expected_accept);
+    else if (params->dtype == PPOW_F32)
+        expected_acceptance_scalar_kernel<float><<<rows, ACC_THREADS, 0, stream>>>(
             (const float *)target_logits, (const float *)draft_logits, valid_len, lse_p, lse_q, K, V, s, expected_accept);
-    } else if (params->dtype == PPOW_F16) {
-        expected_acceptance_kernel<half_bits, false><<<rows, ACC_THREADS, 0, stream>>>(
-            (const half_bits *)target_logits, (const half_bits *)draft_logits, valid_len, lse_p, lse_q, K, V, s,
-            expected_accept);
-    } else if (V % 8 == 0 && (uintptr_t)draft_logits % 16 == 0 && (uintptr_t)target_logits % 16 == 0) {
-        expected_acceptance_kernel<uint16_t, true><<<rows, ACC_THREADS, 0, stream>>>(
-            (const uint16_t *)target_logits, (const uint16_t *)draft_logits, valid_len, lse_p, lse_q, K, V, s,
-            expected_accept);
-    } else {
-        expected_acceptance_kernel<uint16_t, false><<<rows, ACC_THREADS, 0, stream>>>(
-            (const uint16_t *)target_logits, (const uint16_t *)draft_logits, valid_len, lse_p, lse_q, K, V, s,
-            expected_accept);
-    }
+    else if (params->dtype == PPOW_F16)
+        expected_acceptance_scalar_kernel<half_bits><<<rows, ACC_THREADS, 0, stream>>>(
+            (const half_bits *)target_logits, (const half_bits *)draft_logits, valid_len, lse_p, lse_q, K, V, s, expected_accept);
+    else
+        expected_acceptance_scalar_kernel<uint16_t><<<rows, ACC_THREADS, 0, stream>>>(
+            (const uint16_t *)target_logits, (const uint16_t *)draft_logits, valid_len, lse_p, lse_q, K, V, s, expected_accept);
     return cudaGetLastError() == cudaSuccess ? PPOW_OK : PPOW_ERR_CUDA;
 }
 
@@ -450,18 +469,22 @@ extern "C" ppow_status ppow_reference_logprob(const ppow_params *params, const v
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     const float s = (float)(1.4426950408889634074 / (double)params->temperature);
     const unsigned rows = (unsigned)((size_t)params->N * params->K);
-    if (params->dtype == PPOW_F32)
-        reference_logprob_rows_kernel<float, false><<<rows, REF_THREADS, 0, stream>>>(
-            (const float *)ref_target_logits, valid_len, params->K, params->V, s, row_logp);
+    const int32_t K = params->K, V = params->V;
+    const int epu = params->dtype == PPOW_F32 ? 4 : 8;
+    const bool vec = V % epu == 0 && (uintptr_t)ref_target_logits % 16 == 0;
+    const uint4 *ra = (const uint4 *)ref_target_logits;
+    if (vec && params->dtype == PPOW_BF16)
+        reference_logprob_vec_kernel<UnitBf16><<<rows, REF_THREADS, 0, stream>>>(ra, valid_len, K, V / epu, s, row_logp);
+    else if (vec && params->dtype == PPOW_F16)
+        reference_logprob_vec_kernel<UnitF16><<<rows, REF_THREADS, 0, stream>>>(ra, valid_len, K, V / epu, s, row_logp);
+    else if (vec)
+        reference_logprob_vec_kernel<UnitF32><<<rows, REF_THREADS, 0, stream>>>(ra, valid_len, K, V / epu, s, row_logp);
+    else if (params->dtype == PPOW_F32)
+        reference_logprob_scalar_kernel<float><<<rows, REF_THREADS, 0, stream>>>((const float *)ref_target_logits, valid_len, K, V, s, row_logp);
     else if (params->dtype == PPOW_F16)
-        reference_logprob_rows_kernel<half_bits, false><<<rows, REF_THREADS, 0, stream>>>(
-            (const half_bits *)ref_target_logits, valid_len, params->K, params->V, s, row_logp);
-    else if (params->V % 8 == 0 && (uintptr_t)ref_target_logits % 16 == 0)
-        reference_logprob_rows_kernel<uint16_t, true><<<rows, REF_THREADS, 0, stream>>>(
-            (const uint16_t *)ref_target_logits, valid_len, params->K, params->V, s, row_logp);
+        reference_logprob_scalar_kernel<half_bits><<<rows, REF_THREADS, 0, stream>>>((const half_bits *)ref_target_logits, valid_len, K, V, s, row_logp);
     else
-        reference_logprob_rows_kernel<uint16_t, false><<<rows, REF_THREADS, 0, stream>>>(
-            (const uint16_t *)ref_target_logits, valid_len, params->K, params->V, s, row_logp);
+        reference_logprob_scalar_kernel<uint16_t><<<rows, REF_THREADS, 0, stream>>>((const uint16_t *)ref_target_logits, valid_len, K, V, s, row_logp);
     if (cudaGetLastError() != cudaSuccess) return PPOW_ERR_CUDA;
     if (ref_logp) {
         reference_logprob_sum_kernel<<<(unsigned)((params->N + 127) / 128), 128, 0, stream>>>(row_logp, valid_len, params->N,
