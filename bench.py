@@ -222,9 +222,12 @@ def dist_setup(n_gpus):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world > 1:
+    if world > 1 or "RANK" in os.environ:    # launched by torch.distributed.run, even with one rank: use the collective
         import torch.distributed as dist
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29500")
+        os.environ.setdefault("RANK", "0")
+        os.environ.setdefault("WORLD_SIZE", "1")
         backend = "nccl" if torch.cuda.is_available() else "gloo"
         if torch.cuda.is_available():
             torch.cuda.set_device(local)
@@ -380,6 +383,11 @@ def run_reference(args):
 # -------------------------------------------------------------------------------------- ppow arm
 
 
+def _group_is_up():
+    import torch.distributed as dist
+    return dist.is_available() and dist.is_initialized()
+
+
 class Run:
     """One workload resident on the device, with the calls of a step prepared."""
 
@@ -409,7 +417,8 @@ class Run:
         self.score_call = B.ScoreCall(self.params, x["draft_logits"], x["target_logits"], x["draft_tokens"],
                                       x["uniforms"], x["valid_len"], None, self.out, self.ws)
         self.dtype_code = self.params.dtype
-        self.select_call = B.SelectCall(self.out["score"], self.n_keep, self.selected, None, self.sel_ws) if world == 1 else None
+        self.gather = world > 1 or _group_is_up()    # one rank under torch.distributed.run still gathers (same values)
+        self.select_call = None if self.gather else B.SelectCall(self.out["score"], self.n_keep, self.selected, None, self.sel_ws)
         self.acc_events, self.ref_events = [], []
         self.valid_rows = int(x["valid_len"].sum().item()) if x["valid_len"] is not None else N * K
         self.esize = 4 if w.dtype == "f32" else 2
@@ -445,7 +454,7 @@ class Run:
                 ec = torch.cuda.Event(enable_timing=True)
                 ec.record(stream)
                 self.ref_events.append((eb, ec))
-        if self.world > 1:
+        if self.gather:
             scores = self.S.gather_scores(out["score"], self.n_total)    # the one exchange step
             B.ppow_select_windows(scores, self.n_keep, self.selected, None, self.sel_ws, stream)
         else:
@@ -644,7 +653,9 @@ def run_ppow(args):
 
     # ---- one entry per other workload (generated, timed, checked and freed one at a time)
     workloads = None
+    run_gather = run.gather
     launches_per_step, algo_bytes, n_total, n_keep = run.launches_per_step, run.algo_bytes, run.n_total, run.n_keep
+    selected_checksum = int(torch.sum(run.selected.to(torch.int64) * torch.arange(1, n_keep + 1, device=dev)).item()) if n_keep else 0
     if rank == 0 and solo and not args.no_workloads and args.workload == "llama3_like" and not (args.windows or args.logits or args.train):
         run.free()
         workloads = []
@@ -679,7 +690,8 @@ def run_ppow(args):
         "metric": METRIC, "value": value, "unit": "windows/s", "n_gpus": world, "steps": args.steps,
         "warmup": warmup, "ms_per_step": m["step_ms"], "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "storage_dtype": w.dtype, "data": "synthetic",
-        "config": config_of(w, mode), "n_keep_global": n_keep,
+        "config": config_of(w, mode), "n_keep_global": n_keep, "selected_checksum": selected_checksum,
+        "score_exchange": "all_gather over the process group" if run_gather else "none (no process group)",
         "logit_gbs": world * algo_bytes / (m["step_ms"] * 1e-3) / 1e9,
         "roofline": {"bound": "hbm", "kernel": "row_reduce", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
@@ -705,10 +717,9 @@ def main():
         run_reference(args)
     else:
         run_ppow(args)
-    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+    if _group_is_up():
         import torch.distributed as dist
-        if dist.is_initialized():
-            dist.destroy_process_group()
+        dist.destroy_process_group()
 
 
 if __name__ == "__main__":

@@ -48,7 +48,9 @@ typedef enum { PPOW_F32 = 0, PPOW_BF16 = 1, PPOW_F16 = 2 } ppow_dtype;   /* stor
 /* Bits of the device-side error word (ppow_read_error_flags). */
 enum {
     PPOW_FLAG_TOKEN_RANGE = 1u,   /* some draft token was outside [0, V): that position was rejected */
-    PPOW_FLAG_DEVICE_TIMEOUT = 2u /* a bounded wait inside a kernel ran out */
+    PPOW_FLAG_DEVICE_TIMEOUT = 2u, /* a bounded wait inside a kernel ran out */
+    PPOW_FLAG_BOUNDS = 4u          /* bounds-checked build only: an index computed by a kernel was out of range
+                                      (the access was skipped; see ppow_checked_failures) */
 };
 
 typedef struct {
@@ -313,6 +315,19 @@ ppow_status ppow_stream_read_probe(const void *data, size_t bytes, uint32_t *che
 /* Number of kernels one ppow_score_windows call with these parameters launches (1: small problems are scored
  * in a single launch; 2: row reduction + window scan; 0 on invalid parameters).  Launch accounting only. */
 int ppow_score_kernel_launches(const ppow_params *params);
+
+/*
+ * Bounds-checked build (an addition of this library; the paper has no counterpart).  The build script also
+ * produces libppow_checked.so, the same sources compiled with -DPPOW_CHECKED: every index a kernel derives
+ * from N, K, V, the valid lengths, a work item, a tile, a pipeline stage or a token id is tested before use;
+ * a failing test never traps -- it is counted, the access is skipped, and PPOW_FLAG_BOUNDS is set in the
+ * call's error word where there is one.  This call synchronises the device and returns the number of failed
+ * checks since the library was loaded and the site code of the first one (1xx row reduction, 2xx window
+ * scan, 3xx selection, 4xx training side).  In the ordinary library it writes zeros and returns
+ * PPOW_ERR_UNSUPPORTED.
+ *   failures_host     host, required        first_site_host   host or NULL
+ */
+ppow_status ppow_checked_failures(uint32_t *failures_host, uint32_t *first_site_host);
 
 /* Static, never-NULL description of a status code. */
 const char *ppow_status_string(ppow_status status);

@@ -13,7 +13,8 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libppow.so")
+# PPOW_LIBRARY=checked loads the bounds-checked build of the same sources (see ppow_checked_failures)
+LIB_PATH = os.path.join(_HERE, "libppow_checked.so" if os.environ.get("PPOW_LIBRARY") == "checked" else "libppow.so")
 
 PPOW_OK = 0
 PPOW_ERR_INVALID_ARG, PPOW_ERR_UNSUPPORTED, PPOW_ERR_WORKSPACE, PPOW_ERR_CUDA, PPOW_ERR_DEVICE_TIMEOUT = 1, 2, 3, 4, 5
@@ -21,14 +22,14 @@ PPOW_GREEDY, PPOW_STOCHASTIC = 0, 1
 PPOW_F32, PPOW_BF16, PPOW_F16 = 0, 1, 2
 LOGIT_DTYPES = {PPOW_F32: torch.float32, PPOW_BF16: torch.bfloat16, PPOW_F16: torch.float16}
 DTYPE_CODES = {v: k for k, v in LOGIT_DTYPES.items()}
-PPOW_FLAG_TOKEN_RANGE, PPOW_FLAG_DEVICE_TIMEOUT = 1, 2
+PPOW_FLAG_TOKEN_RANGE, PPOW_FLAG_DEVICE_TIMEOUT, PPOW_FLAG_BOUNDS = 1, 2, 4
 
 EXPORTS = ("ppow_score_workspace_bytes", "ppow_score_windows", "ppow_score_windows_traced", "ppow_read_error_flags",
            "ppow_select_workspace_bytes", "ppow_select_windows", "ppow_host_scratch_bytes",
            "ppow_score_and_select_host", "ppow_noalloc_scratch_bytes", "ppow_score_windows_noalloc",
            "ppow_group_advantage", "ppow_sequence_windows", "ppow_sequence_windows_mixed", "ppow_expected_acceptance",
            "ppow_reference_logprob", "ppow_selftest_wait_timeout", "ppow_stream_read_probe", "ppow_score_kernel_launches",
-           "ppow_status_string", "ppow_version")
+           "ppow_checked_failures", "ppow_status_string", "ppow_version")
 
 POSITION_OUTPUTS = {"accept_flag": torch.uint8, "kl": torch.float32, "conf": torch.float32, "crit": torch.float32,
                     "logp_tok": torch.float32, "logq_tok": torch.float32, "target_argmax": torch.int32}
@@ -114,6 +115,8 @@ def load_library():
     lib.ppow_stream_read_probe.argtypes = [vp, sz, vp, vp]
     lib.ppow_score_kernel_launches.restype = ctypes.c_int
     lib.ppow_score_kernel_launches.argtypes = [ctypes.POINTER(ppow_params)]
+    lib.ppow_checked_failures.restype = ctypes.c_int
+    lib.ppow_checked_failures.argtypes = [ctypes.POINTER(ctypes.c_uint32), ctypes.POINTER(ctypes.c_uint32)]
     lib.ppow_status_string.restype = ctypes.c_char_p
     lib.ppow_status_string.argtypes = [ctypes.c_int]
     lib.ppow_version.restype = ctypes.c_int
@@ -169,6 +172,14 @@ def ppow_stream_read_probe(data: torch.Tensor, checksum: torch.Tensor, stream=No
                                     _dev_ptr(checksum, None, "checksum"), _stream_ptr(stream))
     if st != PPOW_OK:
         raise PpowError(st, "ppow_stream_read_probe")
+
+
+def ppow_checked_failures():
+    """(status, failed checks, first failing site) of the bounds-checked build; status PPOW_ERR_UNSUPPORTED and
+    zeros from the ordinary library."""
+    f, site = ctypes.c_uint32(0), ctypes.c_uint32(0)
+    st = load_library().ppow_checked_failures(ctypes.byref(f), ctypes.byref(site))
+    return int(st), int(f.value), int(site.value)
 
 
 def ppow_select_workspace_bytes(N: int) -> int:

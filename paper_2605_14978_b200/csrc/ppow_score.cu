@@ -5,6 +5,7 @@
 #include "../../include/ppow.h"
 #include "ppow_device.cuh"
 #include "ppow_async.cuh"
+#include "ppow_checked.cuh"
 
 #include <math.h>
 
@@ -347,7 +348,11 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
     // copies of P's next tile into stage st
     auto issue = [&](int st) -> int32_t {
         const int32_t n = min(TILE_UNITS, P.u1 - P.u);
-        if (lane == 0) {
+        // the tile lies inside its row, the row inside the tensors, the stage inside the warp's ring
+        if (lane == 0 && PPOW_CHECK(n > 0 && P.u >= 0 && P.u + n <= job.units_per_row && st >= 0 && st < PIPE_STAGES &&
+                                        P.pa + P.u + n <= reinterpret_cast<const uint4 *>(job.target) +
+                                                              (size_t)job.N * job.K * job.units_per_row,
+                                    101, &job.header->error_flags)) {
             const uint32_t bar = bars_addr + 8 * st, dst = stages_addr + st * 2 * TILE_BYTES;
             mbar_arrive_expect_tx(bar, 2u * (uint32_t)n * 16u);
             bulk_load(dst, P.pa + P.u, (uint32_t)n * 16u, bar);
@@ -401,6 +406,7 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
         }
         phases ^= 1u << st;
         pending &= ~(1u << st);
+        if (!PPOW_CHECK(st >= 0 && st < PIPE_STAGES && n > 0 && n <= TILE_UNITS, 104, &job.header->error_flags)) break;
         const uint4 *sa = reinterpret_cast<const uint4 *>(stages + st * 2 * TILE_BYTES);
         const uint4 *sb = reinterpret_cast<const uint4 *>(stages + st * 2 * TILE_BYTES + TILE_BYTES);
         auto refill = [&]() {
@@ -424,7 +430,11 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
             uint4 cand[UNROLL];
 #pragma unroll
             for (int j = 0; j < UNROLL; ++j)
-                if (holder && j < bn) cand[j] = __ldcs(C.pa + bu + j * 32);
+                if (holder && j < bn &&
+                    PPOW_CHECK(bu >= 0 && bu + j * 32 < job.units_per_row, 102, &job.header->error_flags))
+                    cand[j] = __ldcs(C.pa + bu + j * 32);
+                else
+                    cand[j] = Fmt::none();
             RowPartial p = warp_reduce(acc);
             // the consumer moves on to its next item while the re-read is in flight
             const uint32_t done = C.item;
@@ -444,7 +454,7 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
                 }
             }
             arg = warp_min_i32(arg);
-            if (lane == 0) {
+            if (lane == 0 && PPOW_CHECK(done < job.total_items, 103, &job.header->error_flags)) {
                 p.argmax = arg;
                 job.partials[done] = p;
             }
@@ -487,7 +497,7 @@ __global__ void __launch_bounds__(ROW_THREADS, 4) row_reduce_generic_kernel(cons
         const float my_max = acc.max_a;
         RowPartial p = warp_reduce(acc);
         arg = warp_min_i32(my_max == p.max_a ? arg : INT32_MAX);
-        if (lane == 0) {
+        if (lane == 0 && PPOW_CHECK(item < job.total_items && v1 <= job.V && v0 >= 0, 105, &job.header->error_flags)) {
             p.argmax = arg;
             job.partials[item] = p;
         }
@@ -542,14 +552,15 @@ __device__ __forceinline__ void scan_window(const ScanJob &job, const int32_t n,
         // merge this row's partials against the largest references
         double Ra = -INFINITY, Rb = -INFINITY;
         float mx = -INFINITY;
-        for (int i = 0; i < parts; ++i) {
+        const int parts_ok = PPOW_CHECK(parts >= 1 && parts <= (1 << MAX_SHIFT) && pp != nullptr, 201, &job.header->error_flags) ? parts : 0;
+        for (int i = 0; i < parts_ok; ++i) {
             Ra = fmax(Ra, (double)pp[i].rho_a);
             Rb = fmax(Rb, (double)pp[i].rho_b);
             mx = fmaxf(mx, pp[i].max_a);
         }
         double Sa = 0.0, Sb = 0.0, E = 0.0, D = 0.0, Bv = 0.0;
         int32_t arg = INT32_MAX;
-        for (int i = 0; i < parts; ++i) {
+        for (int i = 0; i < parts_ok; ++i) {
             const RowPartial p = pp[i];
             const double da = (double)p.rho_a - Ra, db = (double)p.rho_b - Rb;
             const double fa = exp2(da), fb = exp2(db);
@@ -576,7 +587,9 @@ __device__ __forceinline__ void scan_window(const ScanJob &job, const int32_t n,
 
         const int32_t tok = __ldg(job.tokens + row);
         double lq, lp2 = -INFINITY;
-        if (tok < 0 || tok >= job.V) {
+        if (tok < 0 || tok >= job.V ||
+            !PPOW_CHECK(row < (size_t)job.N * job.K && row * job.V + tok < (size_t)job.N * job.K * job.V, 202,
+                        &job.header->error_flags)) {
             atomicOr(&job.header->error_flags, (unsigned)PPOW_FLAG_TOKEN_RANGE);
             lp = -INFINITY;
             lq = -INFINITY;
@@ -601,7 +614,7 @@ __device__ __forceinline__ void scan_window(const ScanJob &job, const int32_t n,
         o_arg = arg;
     }
 
-    if (lane < K) {
+    if (lane < K && PPOW_CHECK(n >= 0 && n < job.N && K <= 32, 203, &job.header->error_flags)) {
         const size_t row = (size_t)n * K + lane;
         if (job.out.accept_flag) job.out.accept_flag[row] = (uint8_t)flag;
         if (job.out.kl) job.out.kl[row] = o_kl;
@@ -656,6 +669,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
     uint32_t first_part = 0;
     int parts = 0;
     if (lane < job.K) row_items(job.plan, (uint32_t)n * (uint32_t)job.K + (uint32_t)lane, first_part, parts);
+    if (!PPOW_CHECK((size_t)first_part + parts <= job.plan.item_begin[PLAN_CLASSES], 204, &job.header->error_flags)) parts = 0;
     scan_window(job, n, lane, job.partials + first_part, parts);
 }
 
@@ -688,7 +702,7 @@ __global__ void __launch_bounds__(1024) score_small_kernel(const RowJob rj, cons
         const float my_max = acc.max_a;
         RowPartial p = warp_reduce(acc);
         arg = warp_min_i32(my_max == p.max_a ? arg : INT32_MAX);
-        if (lane == 0) {
+        if (lane == 0 && PPOW_CHECK(warp < 32 && row < (size_t)rj.N * rj.K, 106, &rj.header->error_flags)) {
             p.argmax = arg;
             parts[warp] = p;
         }
@@ -957,6 +971,10 @@ extern "C" ppow_status ppow_score_windows(const ppow_params *params,
     return ppow_score_windows_traced(params, draft_logits, target_logits, draft_tokens, uniforms, valid_len,
                                      ref_logp, out, workspace, workspace_bytes, cuda_stream, nullptr, nullptr);
 }
+
+#ifdef PPOW_CHECKED
+namespace ppow { int read_check_counters_score(unsigned int *f, unsigned int *s) { return read_check_counters(f, s); } }
+#endif
 
 extern "C" ppow_status ppow_selftest_wait_timeout(void *workspace, size_t workspace_bytes, uint32_t probes,
                                                   void *cuda_stream)

@@ -9,6 +9,8 @@
 //                     global stage, shared-memory stages fused.
 #include "../../include/ppow.h"
 
+#include "ppow_checked.cuh"
+
 #include <cuda_runtime.h>
 
 namespace ppow {
@@ -49,8 +51,8 @@ __global__ void __launch_bounds__(RANK_THREADS) select_rank_kernel(const float *
         for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
         if (lane == 0) {
             const bool keep = cnt < n_keep;
-            if (keep) selected[cnt] = i;
-            if (mask) mask[i] = keep ? 1 : 0;
+            if (keep && PPOW_CHECK(cnt >= 0 && i < N, 301, nullptr)) selected[cnt] = i;
+            if (mask && PPOW_CHECK(i >= 0 && i < N, 302, nullptr)) mask[i] = keep ? 1 : 0;
         }
     }
 }
@@ -88,7 +90,7 @@ __global__ void __launch_bounds__(SORT_THREADS) sort_local_kernel(unsigned long 
             for (uint32_t t = threadIdx.x; t < SORT_TILE / 2; t += SORT_THREADS) {
                 const uint32_t lo = ((t & ~(j - 1)) << 1) | (t & (j - 1));
                 const bool asc = (((base + lo) & k) == 0);
-                compare_exchange(s[lo], s[lo + j], asc);
+                if (PPOW_CHECK(lo + j < (uint32_t)SORT_TILE, 303, nullptr)) compare_exchange(s[lo], s[lo + j], asc);
             }
             __syncthreads();
         }
@@ -101,6 +103,7 @@ __global__ void sort_global_step_kernel(unsigned long long *__restrict__ keys, u
     const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= n_pad / 2) return;
     const uint32_t lo = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+    if (!PPOW_CHECK(lo + j < n_pad, 304, nullptr)) return;
     unsigned long long a = keys[lo], b = keys[lo + j];
     const bool asc = ((lo & k) == 0);
     if ((a > b) == asc) { keys[lo] = b; keys[lo + j] = a; }
@@ -112,6 +115,7 @@ __global__ void sort_emit_kernel(const unsigned long long *__restrict__ keys, in
     const int32_t r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= N) return;
     const int32_t idx = (int32_t)(keys[r] & 0xffffffffull);
+    if (!PPOW_CHECK(idx >= 0 && idx < N, 305, nullptr)) return;
     if (r < n_keep) selected[r] = idx;
     if (mask) mask[idx] = (r < n_keep) ? 1 : 0;
 }
@@ -179,6 +183,31 @@ extern "C" ppow_status ppow_select_windows(const float *score, int32_t N, int32_
     }
     sort_emit_kernel<<<(N + 255) / 256, 256, 0, stream>>>(keys, N, n_keep, selected, mask);
     return cudaGetLastError() == cudaSuccess ? PPOW_OK : PPOW_ERR_CUDA;
+}
+
+#ifdef PPOW_CHECKED
+namespace ppow {
+int read_check_counters_score(unsigned int *f, unsigned int *s);
+int read_check_counters_train(unsigned int *f, unsigned int *s);
+}
+#endif
+
+extern "C" ppow_status ppow_checked_failures(uint32_t *failures_host, uint32_t *first_site_host)
+{
+    if (!failures_host) return PPOW_ERR_INVALID_ARG;
+#ifdef PPOW_CHECKED
+    unsigned int f = 0, s = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return PPOW_ERR_CUDA;
+    if (read_check_counters(&f, &s) || read_check_counters_score(&f, &s) || read_check_counters_train(&f, &s))
+        return PPOW_ERR_CUDA;
+    *failures_host = f;
+    if (first_site_host) *first_site_host = s;
+    return PPOW_OK;
+#else
+    *failures_host = 0;
+    if (first_site_host) *first_site_host = 0;
+    return PPOW_ERR_UNSUPPORTED;   // not the bounds-checked build
+#endif
 }
 
 extern "C" const char *ppow_status_string(ppow_status status)

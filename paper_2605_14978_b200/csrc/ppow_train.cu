@@ -4,6 +4,7 @@
 // logit tensors a second time.
 #include "../../include/ppow.h"
 #include "ppow_device.cuh"
+#include "ppow_checked.cuh"
 
 #include <math.h>
 
@@ -59,6 +60,7 @@ __global__ void __launch_bounds__(SEQ_THREADS) sequence_windows_kernel(const flo
 
     auto score_of = [&](int32_t j) {
         double sum = 0.0;
+        if (!PPOW_CHECK(j >= 0 && j + K <= T && o0 >= 0, 401, nullptr)) return 0.0;
         for (int32_t t = j; t < j + K; ++t) sum += (double)v[t];
         return sum / (double)K;
     };
@@ -159,6 +161,7 @@ __global__ void __launch_bounds__(ACC_THREADS) expected_acceptance_vec_kernel(co
     const float la = lse_p[row] * 1.4426950408889634f, lb = lse_q[row] * 1.4426950408889634f;
     const uint4 *pa = target + row * (size_t)units, *pb = draft + row * (size_t)units;
     float acc0 = 0.0f, acc1 = 0.0f;
+    if (!PPOW_CHECK(row < (size_t)gridDim.x && k < K, 402, nullptr)) return;
     auto add_unit = [&](const uint4 &A, const uint4 &B) {
         float fa[Unit::EPU], fb[Unit::EPU];
         Unit::unpack(A, fa);
@@ -373,6 +376,10 @@ __global__ void reference_logprob_sum_kernel(const float *__restrict__ row_logp,
 }  // namespace ppow
 
 using namespace ppow;
+
+#ifdef PPOW_CHECKED
+namespace ppow { int read_check_counters_train(unsigned int *f, unsigned int *s) { return read_check_counters(f, s); } }
+#endif
 
 extern "C" ppow_status ppow_group_advantage(const float *reward, int32_t N, int32_t group_size, float delta,
                                             float *advantage, void *cuda_stream)

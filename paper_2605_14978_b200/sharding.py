@@ -67,8 +67,13 @@ def gather_scores(local_score: torch.Tensor, n_total: int, group=None) -> torch.
     width = max(sizes)
     padded = torch.zeros((width,), dtype=local_score.dtype, device=local_score.device)
     padded[: sizes[rank]].copy_(local_score)
-    parts = [torch.empty_like(padded) for _ in range(world)]
-    dist.all_gather(parts, padded, group=group)
+    if local_score.is_cuda:
+        flat = torch.empty((world * width,), dtype=local_score.dtype, device=local_score.device)
+        dist.all_gather_into_tensor(flat, padded, group=group)
+        parts = list(flat.split(width))
+    else:
+        parts = [torch.empty_like(padded) for _ in range(world)]
+        dist.all_gather(parts, padded, group=group)
     return torch.cat([p[:s] for p, s in zip(parts, sizes)])
 
 

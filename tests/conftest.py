@@ -24,3 +24,22 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_sessionfinish(session, exitstatus):
+    """A run against the bounds-checked library (PPOW_LIBRARY=checked) fails if any check failed."""
+    if os.environ.get("PPOW_LIBRARY") != "checked":
+        return
+    try:
+        import torch
+        if not torch.cuda.is_available():
+            return
+        from paper_2605_14978_b200 import binding as B
+        status, failures, site = B.ppow_checked_failures()
+    except Exception as e:                                   # the library could not be asked: that is a failure too
+        print("\nbounds-checked build: could not read the counters: %r" % (e,))
+        session.exitstatus = 3
+        return
+    print("\nbounds-checked build: %d failed checks (status %d, first site %d)" % (failures, status, site))
+    if status != 0 or failures != 0:
+        session.exitstatus = 3
