@@ -117,6 +117,9 @@ size_t ppow_score_workspace_bytes(const ppow_params *params);
  *                                Contents are undefined afterwards except the error word.
  *
  * Returns PPOW_OK once the work is enqueued.  N == 0 is a valid no-op.
+ * If the error word afterwards carries PPOW_FLAG_DEVICE_TIMEOUT (ppow_read_error_flags returns
+ * PPOW_ERR_DEVICE_TIMEOUT), a warp gave up on a bounded wait and left its work items unreduced: every output of
+ * that call is undefined and must be discarded.
  */
 ppow_status ppow_score_windows(const ppow_params *params,
                                const void *draft_logits, const void *target_logits,
@@ -152,9 +155,14 @@ ppow_status ppow_score_windows_traced(const ppow_params *params,
  *     Calls that overlap on the GPU (other streams or host threads) race on it: serialise them.
  *   - The first call on each device looks up the array's device address, which may load the
  *     module: make that first call outside any stream capture.
- *   - The error word of this call cannot be read back with ppow_read_error_flags.
+ *   - The address is remembered per device for the life of the process; do not use this entry point on a
+ *     device whose context the process has destroyed (cudaDeviceReset) since the first call.
+ *   - The error word of the call (out-of-range token, device-side timeout) sits in the shared array: read it
+ *     with ppow_noalloc_read_error_flags (same semantics as ppow_read_error_flags; synchronises the stream)
+ *     before the next call on the device clears it.
  */
 size_t ppow_noalloc_scratch_bytes(void);
+ppow_status ppow_noalloc_read_error_flags(uint32_t *flags_host, void *cuda_stream);
 ppow_status ppow_score_windows_noalloc(const ppow_params *params,
                                        const void *draft_logits, const void *target_logits,
                                        const int32_t *draft_tokens, const float *uniforms,

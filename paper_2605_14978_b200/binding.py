@@ -27,6 +27,7 @@ PPOW_FLAG_TOKEN_RANGE, PPOW_FLAG_DEVICE_TIMEOUT, PPOW_FLAG_BOUNDS = 1, 2, 4
 EXPORTS = ("ppow_score_workspace_bytes", "ppow_score_windows", "ppow_score_windows_traced", "ppow_read_error_flags",
            "ppow_select_workspace_bytes", "ppow_select_windows", "ppow_host_scratch_bytes",
            "ppow_score_and_select_host", "ppow_noalloc_scratch_bytes", "ppow_score_windows_noalloc",
+           "ppow_noalloc_read_error_flags",
            "ppow_group_advantage", "ppow_sequence_windows", "ppow_sequence_windows_mixed", "ppow_expected_acceptance",
            "ppow_reference_logprob", "ppow_selftest_wait_timeout", "ppow_stream_read_probe", "ppow_score_kernel_launches",
            "ppow_checked_failures", "ppow_status_string", "ppow_version")
@@ -99,6 +100,8 @@ def load_library():
     lib.ppow_score_windows_noalloc.restype = ctypes.c_int
     lib.ppow_score_windows_noalloc.argtypes = [ctypes.POINTER(ppow_params), vp, vp, vp, vp, vp, vp,
                                                ctypes.POINTER(ppow_outputs), vp]
+    lib.ppow_noalloc_read_error_flags.restype = ctypes.c_int
+    lib.ppow_noalloc_read_error_flags.argtypes = [ctypes.POINTER(ctypes.c_uint32), vp]
     lib.ppow_group_advantage.restype = ctypes.c_int
     lib.ppow_group_advantage.argtypes = [vp, i32, i32, ctypes.c_float, vp, vp]
     lib.ppow_sequence_windows.restype = ctypes.c_int
@@ -355,6 +358,13 @@ def ppow_score_windows_noalloc(params: ppow_params, draft_logits, target_logits,
         ctypes.byref(o), _stream_ptr(stream))
     if st != PPOW_OK:
         raise PpowError(st, "ppow_score_windows_noalloc")
+
+
+def ppow_noalloc_read_error_flags(stream=None):
+    """(status, flags) left by the last ppow_score_windows_noalloc call on the current device."""
+    flags = ctypes.c_uint32(0)
+    st = load_library().ppow_noalloc_read_error_flags(ctypes.byref(flags), _stream_ptr(stream))
+    return int(st), int(flags.value)
 
 
 def ppow_group_advantage(reward, group_size: int, delta: float, advantage, stream=None) -> None:

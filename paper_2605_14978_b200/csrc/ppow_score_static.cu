@@ -15,7 +15,11 @@
 //     keeps the previous call's contents; the parts that must start at zero (work counter and
 //     error word) are cleared on the stream at the start of every call;
 //   - the first call on each device resolves the array's device address (cudaGetSymbolAddress),
-//     which may load the module; make that first call outside any stream capture.
+//     which may load the module; make that first call outside any stream capture.  The address is
+//     remembered per device ordinal for the life of the process: a process that destroys a device's
+//     context (cudaDeviceReset) must not use this entry point on that device afterwards;
+//   - the call's error word lives at the head of the array: read it with
+//     ppow_noalloc_read_error_flags before the next call on the device overwrites it.
 #include "../../include/ppow.h"
 
 #include <cuda_runtime.h>
@@ -60,9 +64,9 @@ extern "C" ppow_status ppow_score_windows_noalloc(const ppow_params *params,
                                                   const ppow_outputs *out, void *cuda_stream)
 {
     if (!params) return PPOW_ERR_INVALID_ARG;
-    if (params->N == 0) return PPOW_OK;
-    const size_t need = ppow_score_workspace_bytes(params);
+    const size_t need = ppow_score_workspace_bytes(params);   // 0 for parameters the scoring call would refuse
     if (need == 0) return (params->K > 32) ? PPOW_ERR_UNSUPPORTED : PPOW_ERR_INVALID_ARG;
+    if (params->N == 0) return out ? PPOW_OK : PPOW_ERR_INVALID_ARG;
     if (need > PPOW_NOALLOC_SCRATCH_BYTES) return PPOW_ERR_UNSUPPORTED;   // beyond the built-in scratch
     void *scratch = nullptr;
     const ppow_status st = scratch_address(&scratch);
@@ -70,4 +74,15 @@ extern "C" ppow_status ppow_score_windows_noalloc(const ppow_params *params,
     // the scoring call clears the counter and the error word at the head of the workspace itself
     return ppow_score_windows(params, draft_logits, target_logits, draft_tokens, uniforms, valid_len, ref_logp, out,
                               scratch, PPOW_NOALLOC_SCRATCH_BYTES, cuda_stream);
+}
+
+// The error word of the last ppow_score_windows_noalloc call on the current device (it sits at the head of
+// the shared array): same semantics as ppow_read_error_flags, nothing allocated.
+extern "C" ppow_status ppow_noalloc_read_error_flags(uint32_t *flags_host, void *cuda_stream)
+{
+    if (!flags_host) return PPOW_ERR_INVALID_ARG;
+    void *scratch = nullptr;
+    const ppow_status st = scratch_address(&scratch);
+    if (st != PPOW_OK) return st;
+    return ppow_read_error_flags(scratch, flags_host, cuda_stream);
 }

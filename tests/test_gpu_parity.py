@@ -382,6 +382,35 @@ def test_host_buffer_entry_point_with_a_shorter_last_chunk_at_full_vocabulary_wi
     assert len(set(sel_host.tolist()) ^ set(dev_sel.cpu().tolist())) <= 2
 
 
+@pytest.mark.parametrize("T,scale", [(0.7, 8.0), (1.7, 8.0), (0.7, 2.0)])
+def test_uniforms_just_outside_the_band_around_alpha(T, scale):
+    """The kernel scales logits by log2(e)/T rounded to float32, i.e. it evaluates the softmax at T(1 + e) with
+    |e| <= 2^-24; the shift of log alpha is e * (log alpha + H(P) - H(Q)).  Stress: wide logits, T != 1, drafted
+    tokens chosen so that alpha is mid-range -- once the likeliest such token, once the least likely one (90 nats
+    below the mode at scale 8) -- and uniforms placed 1.5e-6 on either side of the oracle's alpha, just outside
+    the band in which flags may differ: every flag must equal the oracle's."""
+    N, K, V = 8, 8, 32000
+    x = _random_inputs(N, K, V, torch.bfloat16, seed=int(10 * T + scale), sigma=1.0, scale=scale)
+    lp = torch.log_softmax(x["target_logits"].double() / T, -1)
+    lq = torch.log_softmax(x["draft_logits"].double() / T, -1)
+    mid = ((lp - lq).exp() > 0.2) & ((lp - lq).exp() < 0.8)
+    picks = {"likely": torch.where(mid, lp, torch.full_like(lp, -1e9)).argmax(-1),
+             "unlikely": torch.where(mid, lp, torch.full_like(lp, 1e9)).argmin(-1)}
+    for name, tok in picks.items():
+        x["draft_tokens"] = tok.to(torch.int32)
+        x["uniforms"] = torch.zeros((N, K), device=DEV)
+        alpha = run_oracle(x, "stochastic", 0.05, T)["alpha"]
+        assert 0.2 < alpha.min() and alpha.max() < 0.8
+        for side in (+1.0, -1.0):
+            u = (alpha + side * 1.5e-6).astype(np.float32)
+            x["uniforms"] = torch.from_numpy(u).to(DEV)
+            gpu = run_gpu(x, "stochastic", 0.05, T)
+            ref = run_oracle(x, "stochastic", 0.05, T)
+            rep = compare_scores(gpu, ref, "stochastic", x["uniforms"])
+            assert rep["band_flag_differences"] == 0, (name, side, rep)
+            assert (ref["accept_flag"] == (side < 0)).all()          # the uniforms sit where they were meant to
+
+
 def test_randomised_shapes_parameters_and_masks():
     """Property-style sweep: seeded random shapes (odd and even V, one position to 32, one window to dozens),
     storage types, temperatures, costs, ragged masks and logit scales; everything is compared with the oracle."""
