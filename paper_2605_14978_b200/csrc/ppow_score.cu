@@ -465,6 +465,37 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
 
 // ---- generic path: any V, any alignment, f32 or bf16 -------------------------------------------
 
+// One warp reduces logits [v0, v1) of a row with scalar coalesced loads: the loads of SCALAR_BATCH strides are
+// issued together (a lane would otherwise have one pair of loads in flight per trip), then folded one by one.
+constexpr int SCALAR_BATCH = 8;
+
+template <typename T, bool REV>
+__device__ __forceinline__ void reduce_span_scalar(const T *pa, const T *pb, int32_t v0, int32_t v1, int lane, float s,
+                                                   RowAcc<REV> &acc, int32_t &arg)
+{
+    for (int32_t base = v0 + lane; base < v1; base += 32 * SCALAR_BATCH) {
+        float a[SCALAR_BATCH], b[SCALAR_BATCH];
+#pragma unroll
+        for (int j = 0; j < SCALAR_BATCH; ++j) {
+            const int32_t v = base + 32 * j;
+            if (v < v1) {
+                a[j] = load_logit<T>(pa, v);
+                b[j] = load_logit<T>(pb, v);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < SCALAR_BATCH; ++j) {
+            const int32_t v = base + 32 * j;
+            if (v < v1) {
+                acc.guard(a[j], b[j], s);
+                if (a[j] > acc.max_a) { acc.max_a = a[j]; arg = v; }   // strict: first occurrence within the lane
+                acc.add_pair(a[j], b[j], s);
+                acc.flush();
+            }
+        }
+    }
+}
+
 template <typename T, bool REV>
 __global__ void __launch_bounds__(ROW_THREADS, 4) row_reduce_generic_kernel(const RowJob job)
 {
@@ -487,13 +518,7 @@ __global__ void __launch_bounds__(ROW_THREADS, 4) row_reduce_generic_kernel(cons
         RowAcc<REV> acc;
         acc.reset();
         int32_t arg = INT32_MAX;
-        for (int32_t v = v0 + lane; v < v1; v += 32) {
-            const float a = load_logit<T>(pa, v), b = load_logit<T>(pb, v);
-            acc.guard(a, b, job.s);
-            if (a > acc.max_a) { acc.max_a = a; arg = v; }   // strict: first occurrence within the lane
-            acc.add_pair(a, b, job.s);
-            acc.flush();
-        }
+        reduce_span_scalar<T, REV>(pa, pb, v0, v1, lane, job.s, acc, arg);
         const float my_max = acc.max_a;
         RowPartial p = warp_reduce(acc);
         arg = warp_min_i32(my_max == p.max_a ? arg : INT32_MAX);
@@ -531,10 +556,63 @@ __device__ __forceinline__ double raw_logit(const void *base, int32_t dtype, siz
 
 constexpr int SCAN_THREADS = 128;
 
-// One warp scores window n, lane = position.  `pp` / `parts`: the partial reductions of this lane's row
-// (unused by lanes beyond the window's valid length).
-__device__ __forceinline__ void scan_window(const ScanJob &job, const int32_t n, const int lane, const RowPartial *pp,
-                                            const int parts)
+// A row's partial reductions merged against the largest references (float64).
+struct RowSums {
+    double Ra, Rb, Sa, Sb, E, D, B;
+    float mx;
+    int32_t arg;
+};
+
+// Contribution of one partial to sums held against the references (Ra, Rb).
+__device__ __forceinline__ void add_partial(RowSums &m, const RowPartial &p)
+{
+    const double da = (double)p.rho_a - m.Ra, db = (double)p.rho_b - m.Rb;
+    const double fa = exp2(da), fb = exp2(db);
+    m.Sa += fa * p.Sa;
+    m.E += fa * (p.E + da * p.Sa);
+    m.D += fa * (p.D + (da - db) * p.Sa);
+    m.Sb += fb * p.Sb;
+    m.B += fb * (p.B + (da - db) * p.Sb);
+    if (p.max_a == m.mx) m.arg = min(m.arg, p.argmax);
+}
+
+// One lane merges all partials of its row, one after the other (rows cut into a few items).
+__device__ __forceinline__ RowSums merge_partials(const RowPartial *pp, int parts)
+{
+    RowSums m = {-INFINITY, -INFINITY, 0.0, 0.0, 0.0, 0.0, 0.0, -INFINITY, INT32_MAX};
+    for (int i = 0; i < parts; ++i) {
+        m.Ra = fmax(m.Ra, (double)pp[i].rho_a);
+        m.Rb = fmax(m.Rb, (double)pp[i].rho_b);
+        m.mx = fmaxf(m.mx, pp[i].max_a);
+    }
+    for (int i = 0; i < parts; ++i) add_partial(m, pp[i]);
+    return m;
+}
+
+// The whole warp merges the partials of one row, lane i taking partial i (rows cut into many items: the
+// last rows of a launch); the result is valid in every lane.
+__device__ __forceinline__ RowSums merge_partials_warp(const RowPartial *pp, int parts, int lane)
+{
+    const bool mine = lane < parts;
+    RowPartial p;
+    if (mine) p = pp[lane];
+    RowSums m = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0f, INT32_MAX};
+    m.Ra = (double)warp_max(mine ? p.rho_a : -INFINITY);
+    m.Rb = (double)warp_max(mine ? p.rho_b : -INFINITY);
+    m.mx = warp_max(mine ? p.max_a : -INFINITY);
+    if (mine) add_partial(m, p);
+    m.Sa = warp_sum_f64(m.Sa);
+    m.Sb = warp_sum_f64(m.Sb);
+    m.E = warp_sum_f64(m.E);
+    m.D = warp_sum_f64(m.D);
+    m.B = warp_sum_f64(m.B);
+    m.arg = warp_min_i32(m.arg);
+    return m;
+}
+
+// One warp scores window n, lane = position.  `m`: the merged reductions of this lane's row (unused by
+// lanes beyond the window's valid length).
+__device__ __forceinline__ void scan_window(const ScanJob &job, const int32_t n, const int lane, const RowSums &m)
 {
     const int32_t K = job.K;
     int32_t L = job.valid_len ? __ldg(job.valid_len + n) : K;
@@ -549,30 +627,9 @@ __device__ __forceinline__ void scan_window(const ScanJob &job, const int32_t n,
 
     if (active) {
         const size_t row = (size_t)n * K + lane;
-        // merge this row's partials against the largest references
-        double Ra = -INFINITY, Rb = -INFINITY;
-        float mx = -INFINITY;
-        const int parts_ok = PPOW_CHECK(parts >= 1 && parts <= (1 << MAX_SHIFT) && pp != nullptr, 201, &job.header->error_flags) ? parts : 0;
-        for (int i = 0; i < parts_ok; ++i) {
-            Ra = fmax(Ra, (double)pp[i].rho_a);
-            Rb = fmax(Rb, (double)pp[i].rho_b);
-            mx = fmaxf(mx, pp[i].max_a);
-        }
-        double Sa = 0.0, Sb = 0.0, E = 0.0, D = 0.0, Bv = 0.0;
-        int32_t arg = INT32_MAX;
-        for (int i = 0; i < parts_ok; ++i) {
-            const RowPartial p = pp[i];
-            const double da = (double)p.rho_a - Ra, db = (double)p.rho_b - Rb;
-            const double fa = exp2(da), fb = exp2(db);
-            const double pSa = p.Sa, pSb = p.Sb;
-            const double sa = fa * pSa;
-            Sa += sa;
-            E += fa * (p.E + da * pSa);
-            D += fa * (p.D + (da - db) * pSa);
-            Sb += fb * pSb;
-            Bv += fb * (p.B + (da - db) * pSb);
-            if (p.max_a == mx) arg = min(arg, p.argmax);
-        }
+        const double Ra = m.Ra, Rb = m.Rb, Sa = m.Sa, Sb = m.Sb, E = m.E, D = m.D, Bv = m.B;
+        const float mx = m.mx;
+        const int32_t arg = m.arg;
         const double s = (double)job.s;
         const double l2Sa = log2(Sa), l2Sb = log2(Sb);
         const double H = (l2Sa - E / Sa) * LN2;                 // entropy of P, nats
@@ -668,9 +725,27 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
     if (n >= job.N) return;
     uint32_t first_part = 0;
     int parts = 0;
-    if (lane < job.K) row_items(job.plan, (uint32_t)n * (uint32_t)job.K + (uint32_t)lane, first_part, parts);
-    if (!PPOW_CHECK((size_t)first_part + parts <= job.plan.item_begin[PLAN_CLASSES], 204, &job.header->error_flags)) parts = 0;
-    scan_window(job, n, lane, job.partials + first_part, parts);
+    int32_t L = job.valid_len ? __ldg(job.valid_len + n) : job.K;
+    L = max(0, min(L, job.K));
+    if (lane < L) row_items(job.plan, (uint32_t)n * (uint32_t)job.K + (uint32_t)lane, first_part, parts);
+    if (!PPOW_CHECK((size_t)first_part + parts <= job.plan.item_begin[PLAN_CLASSES] && parts <= (1 << MAX_SHIFT), 204,
+                    &job.header->error_flags))
+        parts = 0;
+    RowSums m = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0f, INT32_MAX};
+    int most = parts;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) most = max(most, __shfl_xor_sync(0xffffffffu, most, o));
+    if (most <= 4) {
+        if (lane < L) m = merge_partials(job.partials + first_part, parts);
+    } else {   // rows near the end of the launch: up to 32 partials each, merged by the whole warp row by row
+        for (int r = 0; r < L; ++r) {
+            const uint32_t fp = __shfl_sync(0xffffffffu, first_part, r);
+            const int np = __shfl_sync(0xffffffffu, parts, r);
+            const RowSums mr = merge_partials_warp(job.partials + fp, np, lane);
+            if (lane == r) m = mr;
+        }
+    }
+    scan_window(job, n, lane, m);
 }
 
 // ---- small problems: the whole pass in one launch ---------------------------------------------------
@@ -692,13 +767,7 @@ __global__ void __launch_bounds__(1024) score_small_kernel(const RowJob rj, cons
         RowAcc<REV> acc;
         acc.reset();
         int32_t arg = INT32_MAX;
-        for (int32_t v = lane; v < rj.V; v += 32) {
-            const float a = load_logit<T>(pa, v), b = load_logit<T>(pb, v);
-            acc.guard(a, b, rj.s);
-            if (a > acc.max_a) { acc.max_a = a; arg = v; }   // strict: first occurrence within the lane
-            acc.add_pair(a, b, rj.s);
-            acc.flush();
-        }
+        reduce_span_scalar<T, REV>(pa, pb, 0, rj.V, lane, rj.s, acc, arg);
         const float my_max = acc.max_a;
         RowPartial p = warp_reduce(acc);
         arg = warp_min_i32(my_max == p.max_a ? arg : INT32_MAX);
@@ -708,7 +777,7 @@ __global__ void __launch_bounds__(1024) score_small_kernel(const RowJob rj, cons
         }
     }
     __syncthreads();
-    if (warp == 0) scan_window(sj, n, lane, &parts[lane < rj.K ? lane : 0], 1);
+    if (warp == 0) scan_window(sj, n, lane, merge_partials(&parts[lane < rj.K ? lane : 0], lane < L ? 1 : 0));
 }
 
 // ---- self-test of the bounded wait ----------------------------------------------------------------

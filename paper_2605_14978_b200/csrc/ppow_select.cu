@@ -13,6 +13,8 @@
 
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 namespace ppow {
 
 constexpr int RANK_MAX_N = 16384;
@@ -153,18 +155,28 @@ extern "C" ppow_status ppow_select_windows(const float *score, int32_t N, int32_
         return PPOW_OK;
     }
     if (N <= RANK_MAX_N) {
-        int dev = 0, sms = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            return PPOW_ERR_CUDA;
+        // launch limits of the device, looked up once (host calls of a few microseconds each)
+        static std::atomic<int> sms_of[64];
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return PPOW_ERR_CUDA;
+        int sms = (dev >= 0 && dev < 64) ? sms_of[dev].load(std::memory_order_relaxed) : 0;
+        if (sms <= 0) {
+            if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+                return PPOW_ERR_CUDA;
+            if (cudaFuncSetAttribute(select_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     RANK_MAX_N * (int)sizeof(uint32_t)) != cudaSuccess)
+                return PPOW_ERR_CUDA;
+            if (dev >= 0 && dev < 64) sms_of[dev].store(sms, std::memory_order_relaxed);
+        }
         const size_t smem = (size_t)N * sizeof(uint32_t);
-        if (smem > 48 * 1024 &&
-            cudaFuncSetAttribute(select_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-            return PPOW_ERR_CUDA;
         int grid = (N + (RANK_THREADS / 32) - 1) / (RANK_THREADS / 32);
         if (grid > sms * 4) grid = sms * 4;
         select_rank_kernel<<<grid, RANK_THREADS, smem, stream>>>(score, N, n_keep, selected, mask);
-        return cudaGetLastError() == cudaSuccess ? PPOW_OK : PPOW_ERR_CUDA;
+        if (cudaGetLastError() != cudaSuccess) {
+            if (dev >= 0 && dev < 64) sms_of[dev].store(0, std::memory_order_relaxed);   // look the limits up again next time
+            return PPOW_ERR_CUDA;
+        }
+        return PPOW_OK;
     }
 
     const size_t need = ppow_select_workspace_bytes(N);
