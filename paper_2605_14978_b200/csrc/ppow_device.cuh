@@ -31,6 +31,18 @@ __device__ __forceinline__ float f16_to_f32(uint16_t bits) { return __half2float
 constexpr float REBASE_LOG2 = 4.0f;      // raise a reference when a tile exceeds it by 2^4
 constexpr float RHO_INIT = -1.0e30f;     // "no reference yet": the first tile always rebases
 
+// References are whole numbers (log2 units), so moving a sum from one reference to another multiplies it by an
+// exact power of two: no rounding in rebase(), none when partial sums of a row are merged.
+// 2^d for a whole number d <= 0 (0 below the normal range: the sum it scales is negligible there).
+__device__ __forceinline__ float pow2_whole(float d)
+{
+    return d < -126.0f ? 0.0f : __int_as_float((127 + (int)d) << 23);
+}
+__device__ __forceinline__ double pow2_whole(double d)
+{
+    return d < -1022.0 ? 0.0 : __longlong_as_double((long long)(1023 + (int)d) << 52);
+}
+
 // One partial reduction of (part of) a row; merged later in float64.
 struct __align__(16) RowPartial {
     float rho_a, rho_b;   // references, log2 units
@@ -119,7 +131,7 @@ struct RowAcc {
     {
         const float da = rho_a - new_rho_a, db = rho_b - new_rho_b;
         if (da == 0.0f && db == 0.0f) return;
-        const float fa = ex2_approx(da), fb = ex2_approx(db);
+        const float fa = pow2_whole(da), fb = pow2_whole(db);   // exact: references are whole numbers
         const float S = Sa_hi + Sa_lo;
         Et = fa * fmaf(da, S, Et);
         Dt = fa * fmaf(da - db, S, Dt);
@@ -174,7 +186,7 @@ struct RowAcc {
     {
         const bool up_a = fmaf(tile_max_a, s, -rho_a) > REBASE_LOG2;
         const bool up_b = fmaf(tile_max_b, s, -rho_b) > REBASE_LOG2;
-        if (up_a | up_b) rebase(up_a ? tile_max_a * s : rho_a, up_b ? tile_max_b * s : rho_b);
+        if (up_a | up_b) rebase(up_a ? ceilf(tile_max_a * s) : rho_a, up_b ? ceilf(tile_max_b * s) : rho_b);
     }
 };
 

@@ -563,51 +563,63 @@ struct RowSums {
     int32_t arg;
 };
 
-// Contribution of one partial to sums held against the references (Ra, Rb).
-__device__ __forceinline__ void add_partial(RowSums &m, const RowPartial &p)
+// Folds the sums `p` of one part of a row into `m`, carrying the larger references: moving either side to a new
+// reference is a multiplication by an exact power of two (references are whole numbers), so the order of the
+// parts only matters to the rounding of the float64 additions.  A side that holds nothing (Sa == 0: every
+// real part has a term near 2^0) is skipped.
+__device__ __forceinline__ void fold_sums(RowSums &m, const RowSums &p)
 {
-    const double da = (double)p.rho_a - m.Ra, db = (double)p.rho_b - m.Rb;
-    const double fa = exp2(da), fb = exp2(db);
-    m.Sa += fa * p.Sa;
-    m.E += fa * (p.E + da * p.Sa);
-    m.D += fa * (p.D + (da - db) * p.Sa);
-    m.Sb += fb * p.Sb;
-    m.B += fb * (p.B + (da - db) * p.Sb);
-    if (p.max_a == m.mx) m.arg = min(m.arg, p.argmax);
-}
-
-// One lane merges all partials of its row, one after the other (rows cut into a few items).
-__device__ __forceinline__ RowSums merge_partials(const RowPartial *pp, int parts)
-{
-    RowSums m = {-INFINITY, -INFINITY, 0.0, 0.0, 0.0, 0.0, 0.0, -INFINITY, INT32_MAX};
-    for (int i = 0; i < parts; ++i) {
-        m.Ra = fmax(m.Ra, (double)pp[i].rho_a);
-        m.Rb = fmax(m.Rb, (double)pp[i].rho_b);
-        m.mx = fmaxf(m.mx, pp[i].max_a);
+    if (p.Sa == 0.0) return;
+    if (m.Sa == 0.0) {
+        m = p;
+        return;
     }
-    for (int i = 0; i < parts; ++i) add_partial(m, pp[i]);
+    const double Ra = fmax(m.Ra, p.Ra), Rb = fmax(m.Rb, p.Rb);
+    const double da0 = m.Ra - Ra, db0 = m.Rb - Rb;   // what is held so far: one of each pair is 0
+    const double da1 = p.Ra - Ra, db1 = p.Rb - Rb;   // the new part
+    const double fa0 = pow2_whole(da0), fb0 = pow2_whole(db0), fa1 = pow2_whole(da1), fb1 = pow2_whole(db1);
+    m.E = fa0 * (m.E + da0 * m.Sa) + fa1 * (p.E + da1 * p.Sa);
+    m.D = fa0 * (m.D + (da0 - db0) * m.Sa) + fa1 * (p.D + (da1 - db1) * p.Sa);
+    m.B = fb0 * (m.B + (da0 - db0) * m.Sb) + fb1 * (p.B + (da1 - db1) * p.Sb);
+    m.Sa = fa0 * m.Sa + fa1 * p.Sa;
+    m.Sb = fb0 * m.Sb + fb1 * p.Sb;
+    m.Ra = Ra;
+    m.Rb = Rb;
+    m.arg = p.mx > m.mx ? p.arg : (p.mx == m.mx ? min(m.arg, p.arg) : m.arg);
+    m.mx = fmaxf(m.mx, p.mx);
+}
+
+__device__ __forceinline__ RowSums sums_of(const RowPartial &p)
+{
+    RowSums r = {(double)p.rho_a, (double)p.rho_b, p.Sa, p.Sb, p.E, p.D, p.B, p.max_a, p.argmax};
+    return r;
+}
+
+// One lane merges parts start, start + stride, ... of a row, four loads at a time (a lane would otherwise
+// wait for memory once per part).
+__device__ __forceinline__ RowSums merge_partials(const RowPartial *pp, int parts, int start = 0, int stride = 1)
+{
+    RowSums m = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, -INFINITY, INT32_MAX};
+    for (int i0 = start; i0 < parts; i0 += 4 * stride) {
+        RowPartial q[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (i0 + j * stride < parts) q[j] = pp[i0 + j * stride];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (i0 + j * stride < parts) fold_sums(m, sums_of(q[j]));
+    }
     return m;
 }
 
-// The whole warp merges the partials of one row, lane i taking partial i (rows cut into many items: the
-// last rows of a launch); the result is valid in every lane.
-__device__ __forceinline__ RowSums merge_partials_warp(const RowPartial *pp, int parts, int lane)
+__device__ __forceinline__ RowSums shfl_sums(const RowSums &m, int src_lane, bool xor_mode)
 {
-    const bool mine = lane < parts;
-    RowPartial p;
-    if (mine) p = pp[lane];
-    RowSums m = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0f, INT32_MAX};
-    m.Ra = (double)warp_max(mine ? p.rho_a : -INFINITY);
-    m.Rb = (double)warp_max(mine ? p.rho_b : -INFINITY);
-    m.mx = warp_max(mine ? p.max_a : -INFINITY);
-    if (mine) add_partial(m, p);
-    m.Sa = warp_sum_f64(m.Sa);
-    m.Sb = warp_sum_f64(m.Sb);
-    m.E = warp_sum_f64(m.E);
-    m.D = warp_sum_f64(m.D);
-    m.B = warp_sum_f64(m.B);
-    m.arg = warp_min_i32(m.arg);
-    return m;
+    RowSums r;
+#define PPOW_SH(x) (xor_mode ? __shfl_xor_sync(0xffffffffu, (x), src_lane) : __shfl_sync(0xffffffffu, (x), src_lane))
+    r.Ra = PPOW_SH(m.Ra); r.Rb = PPOW_SH(m.Rb); r.Sa = PPOW_SH(m.Sa); r.Sb = PPOW_SH(m.Sb);
+    r.E = PPOW_SH(m.E); r.D = PPOW_SH(m.D); r.B = PPOW_SH(m.B); r.mx = PPOW_SH(m.mx); r.arg = PPOW_SH(m.arg);
+#undef PPOW_SH
+    return r;
 }
 
 // One warp scores window n, lane = position.  `m`: the merged reductions of this lane's row (unused by
@@ -727,24 +739,19 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
     int parts = 0;
     int32_t L = job.valid_len ? __ldg(job.valid_len + n) : job.K;
     L = max(0, min(L, job.K));
-    if (lane < L) row_items(job.plan, (uint32_t)n * (uint32_t)job.K + (uint32_t)lane, first_part, parts);
+    // G lanes share the merge of one row's parts (rows near the end of the launch are cut into up to 32 items):
+    // lanes [r*G, r*G + G) take parts sub, sub + G, ... of row r, fold their results together, and lane t, which
+    // scores position t, fetches row t's sums from lane t*G
+    int kp = 1;
+    while (kp < job.K) kp <<= 1;
+    const int G = 32 / kp, r = lane / G, sub = lane & (G - 1);
+    if (r < L) row_items(job.plan, (uint32_t)n * (uint32_t)job.K + (uint32_t)r, first_part, parts);
     if (!PPOW_CHECK((size_t)first_part + parts <= job.plan.item_begin[PLAN_CLASSES] && parts <= (1 << MAX_SHIFT), 204,
                     &job.header->error_flags))
         parts = 0;
-    RowSums m = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0f, INT32_MAX};
-    int most = parts;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) most = max(most, __shfl_xor_sync(0xffffffffu, most, o));
-    if (most <= 4) {
-        if (lane < L) m = merge_partials(job.partials + first_part, parts);
-    } else {   // rows near the end of the launch: up to 32 partials each, merged by the whole warp row by row
-        for (int r = 0; r < L; ++r) {
-            const uint32_t fp = __shfl_sync(0xffffffffu, first_part, r);
-            const int np = __shfl_sync(0xffffffffu, parts, r);
-            const RowSums mr = merge_partials_warp(job.partials + fp, np, lane);
-            if (lane == r) m = mr;
-        }
-    }
+    RowSums m = merge_partials(job.partials + first_part, parts, sub, G);
+    for (int o = G >> 1; o > 0; o >>= 1) fold_sums(m, shfl_sums(m, o, true));
+    m = shfl_sums(m, (lane * G) & 31, false);
     scan_window(job, n, lane, m);
 }
 
