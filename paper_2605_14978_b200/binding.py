@@ -14,7 +14,9 @@ import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 # PPOW_LIBRARY=checked loads the bounds-checked build of the same sources (see ppow_checked_failures)
-LIB_PATH = os.path.join(_HERE, "libppow_checked.so" if os.environ.get("PPOW_LIBRARY") == "checked" else "libppow.so")
+#                        timeline loads the build whose row kernel records a per-warp timeline (ppow_timeline_read)
+LIB_PATH = os.path.join(_HERE, {"checked": "libppow_checked.so", "timeline": "libppow_timeline.so"}.get(
+    os.environ.get("PPOW_LIBRARY", ""), "libppow.so"))
 
 PPOW_OK = 0
 PPOW_ERR_INVALID_ARG, PPOW_ERR_UNSUPPORTED, PPOW_ERR_WORKSPACE, PPOW_ERR_CUDA, PPOW_ERR_DEVICE_TIMEOUT = 1, 2, 3, 4, 5
@@ -30,7 +32,7 @@ EXPORTS = ("ppow_score_workspace_bytes", "ppow_score_windows", "ppow_score_windo
            "ppow_noalloc_read_error_flags",
            "ppow_group_advantage", "ppow_sequence_windows", "ppow_sequence_windows_mixed", "ppow_expected_acceptance",
            "ppow_reference_logprob", "ppow_selftest_wait_timeout", "ppow_stream_read_probe", "ppow_score_kernel_launches",
-           "ppow_checked_failures", "ppow_status_string", "ppow_version")
+           "ppow_checked_failures", "ppow_timeline_read", "ppow_status_string", "ppow_version")
 
 POSITION_OUTPUTS = {"accept_flag": torch.uint8, "kl": torch.float32, "conf": torch.float32, "crit": torch.float32,
                     "logp_tok": torch.float32, "logq_tok": torch.float32, "target_argmax": torch.int32}
@@ -120,6 +122,8 @@ def load_library():
     lib.ppow_score_kernel_launches.argtypes = [ctypes.POINTER(ppow_params)]
     lib.ppow_checked_failures.restype = ctypes.c_int
     lib.ppow_checked_failures.argtypes = [ctypes.POINTER(ctypes.c_uint32), ctypes.POINTER(ctypes.c_uint32)]
+    lib.ppow_timeline_read.restype = ctypes.c_int
+    lib.ppow_timeline_read.argtypes = [vp, sz]
     lib.ppow_status_string.restype = ctypes.c_char_p
     lib.ppow_status_string.argtypes = [ctypes.c_int]
     lib.ppow_version.restype = ctypes.c_int
@@ -183,6 +187,14 @@ def ppow_checked_failures():
     f, site = ctypes.c_uint32(0), ctypes.c_uint32(0)
     st = load_library().ppow_checked_failures(ctypes.byref(f), ctypes.byref(site))
     return int(st), int(f.value), int(site.value)
+
+
+def ppow_timeline_read(warps: int):
+    """(status, array [warps, 9] of uint64) from the timeline build; status PPOW_ERR_UNSUPPORTED otherwise."""
+    import numpy as np
+    buf = np.zeros((int(warps), 9), dtype=np.uint64)
+    st = load_library().ppow_timeline_read(ctypes.c_void_p(buf.ctypes.data), int(warps))
+    return int(st), buf
 
 
 def ppow_select_workspace_bytes(N: int) -> int:

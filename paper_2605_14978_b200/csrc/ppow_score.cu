@@ -13,6 +13,30 @@
 
 namespace ppow {
 
+// Timeline build (-DPPOW_TIMELINE): every warp of the bulk-copy kernel leaves eight 64-bit words behind --
+// start, first data and end (%globaltimer, ns), items and tiles done, SM id, cycles spent waiting for copies,
+// cycles spent in item ends -- plus its total cycles; ppow_timeline_read copies them out.  Costs a few
+// instructions per tile; the ordinary build has none of it.
+#ifdef PPOW_TIMELINE
+constexpr int TIMELINE_WARPS = 4096;
+__device__ unsigned long long g_timeline[TIMELINE_WARPS * 9];
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ unsigned sm_id()
+{
+    unsigned t;
+    asm volatile("mov.u32 %0, %smid;" : "=r"(t));
+    return t;
+}
+#define PPOW_TL(...) __VA_ARGS__
+#else
+#define PPOW_TL(...)
+#endif
+
 constexpr int ROW_THREADS = 256;   // threads per CTA of the scalar row-reduction kernels
 constexpr int UNROLL = 4;          // 16-byte units per lane per tensor in one tile (< 8: packed with the unit index)
 constexpr int TILE_UNITS = 32 * UNROLL;       // 16-byte units per tile per tensor
@@ -320,6 +344,8 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
     __shared__ uint32_t item_ring[PIPE_WARPS][ITEM_RING];
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    PPOW_TL(const unsigned long long tl_t0 = global_ns(); unsigned long long tl_t1 = 0; unsigned tl_items = 0, tl_tiles = 0;
+            long long tl_wait = 0, tl_end = 0; const long long tl_c0 = clock64();)
     unsigned char *stages = pipe_smem + (size_t)warp * PIPE_STAGES * 2 * TILE_BYTES;
     const uint32_t stages_addr = smem_addr(stages);
     const uint32_t bars_addr = smem_addr(&full_bar[warp][0]);
@@ -396,7 +422,10 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
         const int32_t n = min(TILE_UNITS, C.u1 - C.u);
         // every lane waits (the tile becomes visible to the lanes that observed the phase); the vote keeps
         // the warp together if the limit is hit by only some of them
-        if (!__all_sync(0xffffffffu, mbar_wait_bounded(bars_addr + 8 * st, (phases >> st) & 1u, WAIT_LIMIT))) {
+        PPOW_TL(const long long tl_w0 = clock64();)
+        const bool arrived = __all_sync(0xffffffffu, mbar_wait_bounded(bars_addr + 8 * st, (phases >> st) & 1u, WAIT_LIMIT));
+        PPOW_TL(tl_wait += clock64() - tl_w0; if (tl_t1 == 0) tl_t1 = global_ns(); ++tl_tiles;)
+        if (!arrived) {
             // give up: report, wait (bounded) for the copies still aimed at this warp's stages, leave
             if (lane == 0) atomicOr(&job.header->error_flags, (unsigned)PPOW_FLAG_DEVICE_TIMEOUT);
 #pragma unroll
@@ -420,6 +449,7 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
         C.u += n;
 
         if (C.u >= C.u1) {   // end of the item: warp reduction, argmax index, one partial
+            PPOW_TL(const long long tl_e0 = clock64();)
             // The lanes that hold the item's maximum re-read the units of the tile that raised it, to find the
             // lowest vocabulary index.  The loads are issued as soon as the maximum is known, so that the rest
             // of the warp reduction covers their latency.
@@ -458,9 +488,16 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
                 p.argmax = arg;
                 job.partials[done] = p;
             }
+            PPOW_TL(++tl_items; tl_end += clock64() - tl_e0;)
         }
         st = (st + 1 == PIPE_STAGES) ? 0 : st + 1;
     }
+    PPOW_TL(const unsigned tl_w = blockIdx.x * PIPE_WARPS + warp;
+            if (lane == 0 && tl_w < TIMELINE_WARPS) {
+                unsigned long long *o = g_timeline + (size_t)tl_w * 9;
+                o[0] = tl_t0; o[1] = tl_t1; o[2] = global_ns(); o[3] = tl_items; o[4] = tl_tiles; o[5] = sm_id();
+                o[6] = (unsigned long long)tl_wait; o[7] = (unsigned long long)tl_end; o[8] = (unsigned long long)(clock64() - tl_c0);
+            })
 }
 
 // ---- generic path: any V, any alignment, f32 or bf16 -------------------------------------------
@@ -1051,6 +1088,19 @@ extern "C" ppow_status ppow_score_windows(const ppow_params *params,
 #ifdef PPOW_CHECKED
 namespace ppow { int read_check_counters_score(unsigned int *f, unsigned int *s) { return read_check_counters(f, s); } }
 #endif
+
+extern "C" ppow_status ppow_timeline_read(uint64_t *words_host, size_t warps)
+{
+    if (!words_host) return PPOW_ERR_INVALID_ARG;
+#ifdef PPOW_TIMELINE
+    if (warps > (size_t)TIMELINE_WARPS) return PPOW_ERR_INVALID_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return PPOW_ERR_CUDA;
+    return cudaMemcpyFromSymbol(words_host, g_timeline, warps * 9 * sizeof(unsigned long long)) == cudaSuccess ? PPOW_OK : PPOW_ERR_CUDA;
+#else
+    (void)warps;
+    return PPOW_ERR_UNSUPPORTED;   // not the timeline build
+#endif
+}
 
 extern "C" ppow_status ppow_selftest_wait_timeout(void *workspace, size_t workspace_bytes, uint32_t probes,
                                                   void *cuda_stream)

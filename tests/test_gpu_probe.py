@@ -1,4 +1,8 @@
 """Measurement aids of the library: the read-only streaming probe and the launch-count query."""
+import os
+import subprocess
+import sys
+
 import numpy as np
 import pytest
 import torch
@@ -27,3 +31,14 @@ def test_launch_count_query_names_the_one_launch_path():
     assert B.ppow_score_kernel_launches(B.make_params(2048, 8, 128256, B.PPOW_BF16, B.PPOW_STOCHASTIC, 0.04)) == 2
     assert B.ppow_score_kernel_launches(B.make_params(132, 4, 1000, B.PPOW_F32, B.PPOW_GREEDY, 0.05)) == 2
     assert B.ppow_score_kernel_launches(B.make_params(64, 40, 1000, B.PPOW_F32, B.PPOW_GREEDY, 0.05)) == 0
+
+
+def test_timeline_build_records_every_warp_and_the_ordinary_library_declines():
+    status, _ = B.ppow_timeline_read(8)
+    assert status == B.PPOW_ERR_UNSUPPORTED
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, PPOW_LIBRARY="timeline")
+    res = subprocess.run([sys.executable, "-m", "paper_2605_14978_b200.timeline", "llama3_like:64"], capture_output=True,
+                         text=True, timeout=900, env=env, cwd=root)
+    assert res.returncode == 0, res.stderr[-2000:]
+    assert "== llama3_like:64: 2368 warps" in res.stdout and "start to first data" in res.stdout, res.stdout[-2000:]
