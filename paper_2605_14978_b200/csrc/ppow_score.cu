@@ -73,8 +73,11 @@ struct RowJob {
     WsHeader *header;
     WorkPlan plan;
     int32_t N, K, V;
-    int32_t units_per_row;     // 16-byte units per row (bulk-copy kernel only)
+    int32_t units_per_row;     // 16-byte units per row (bulk-copy kernel, rows of whole aligned units)
     int32_t tile_logits;       // logits per tile (scalar kernel: item boundaries in logits)
+    int32_t shifted;           // bulk-copy kernel: rows are not whole 16-byte aligned units (odd V or an offset base)
+    int32_t es_shift;          // log2 of the bytes per logit
+    int64_t row_bytes;         // bytes per row
     uint32_t total_items;
     float s;                   // log2(e)/T
 };
@@ -182,25 +185,42 @@ constexpr size_t PIPE_SMEM_BYTES = (size_t)PIPE_WARPS * PIPE_STAGES * 2 * TILE_B
 
 struct ItemCursor {
     uint32_t item;          // >= total_items: nothing left
-    int32_t u, u1;          // next unit and end of the item, relative to the row
-    const uint4 *pa, *pb;   // row bases
+    int32_t u, u1;          // next unit and end of the item, relative to the row's first unit
+    int32_t units, head;    // units the row spans; logits of its first unit that belong to the row before (0 unless shifted)
+    const uint4 *pa, *pb;   // first unit of the row in each tensor (16-byte aligned)
 };
 
 __device__ __forceinline__ void open_item(const RowJob &job, ItemCursor &c, uint32_t item)
 {
     c.item = item;
     c.u = c.u1 = 0;
+    c.units = c.head = 0;
     c.pa = c.pb = nullptr;
     if (item >= job.total_items) return;
-    const int32_t units_per_row = job.units_per_row;
     uint32_t row;
     int32_t t0, t1;
     locate_item(job.plan, item, row, t0, t1);
+    if (!job.shifted) {
+        c.units = job.units_per_row;
+        c.pa = reinterpret_cast<const uint4 *>(job.target) + (size_t)row * c.units;
+        c.pb = reinterpret_cast<const uint4 *>(job.draft) + (size_t)row * c.units;
+    } else {
+        // A row that starts inside a 16-byte unit: the units are taken from the aligned address below its
+        // start (both tensors have the same offset), `head` logits of the first unit and the logits past the
+        // row's end in the last one are masked out when those units are read.
+        const uintptr_t a = reinterpret_cast<uintptr_t>(job.target) + (size_t)row * (size_t)job.row_bytes;
+        const uintptr_t b = reinterpret_cast<uintptr_t>(job.draft) + (size_t)row * (size_t)job.row_bytes;
+        const int epu_shift = 4 - job.es_shift;
+        c.head = (int32_t)((a & 15u) >> job.es_shift);
+        c.units = (c.head + job.V + (1 << epu_shift) - 1) >> epu_shift;
+        c.pa = reinterpret_cast<const uint4 *>(a & ~(uintptr_t)15);
+        c.pb = reinterpret_cast<const uint4 *>(b & ~(uintptr_t)15);
+    }
     c.u = t0 * TILE_UNITS;
-    c.u1 = min(t1 * TILE_UNITS, units_per_row);
-    c.pa = reinterpret_cast<const uint4 *>(job.target) + (size_t)row * units_per_row;
-    c.pb = reinterpret_cast<const uint4 *>(job.draft) + (size_t)row * units_per_row;
+    c.u1 = (t1 == job.plan.tiles) ? c.units : t1 * TILE_UNITS;   // the last item of a row takes what is left of it
 }
+
+__device__ __forceinline__ void mask_halves(uint4 &w4, int lo, int hi, uint32_t bits);
 
 // Storage formats of the bulk-copy kernel: how a 16-byte unit of logits is read.
 struct FmtBf16 {
@@ -238,7 +258,21 @@ struct FmtBf16 {
         }
         return pos;
     }
+    // logits outside [lo, hi) of the unit do not belong to the row: replaced by a finite, hugely negative value
+    // (-1e25: its term 2^x is 0 and 0 * x stays 0, which -inf would not)
+    static __device__ __forceinline__ void mask_unit(uint4 &w4, int lo, int hi) { mask_halves(w4, lo, hi, 0xe904u); }
 };
+
+__device__ __forceinline__ void mask_halves(uint4 &w4, int lo, int hi, uint32_t bits)
+{
+    uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        if (2 * q < lo || 2 * q >= hi) w[q] = (w[q] & 0xffff0000u) | bits;
+        if (2 * q + 1 < lo || 2 * q + 1 >= hi) w[q] = (w[q] & 0x0000ffffu) | (bits << 16);
+    }
+    w4 = make_uint4(w[0], w[1], w[2], w[3]);
+}
 
 struct FmtF16 {
     static constexpr int EPU = 8;
@@ -274,6 +308,7 @@ struct FmtF16 {
         }
         return pos;
     }
+    static __device__ __forceinline__ void mask_unit(uint4 &w4, int lo, int hi) { mask_halves(w4, lo, hi, 0xfbffu); }   // -65504
 };
 
 struct FmtF32 {
@@ -306,13 +341,33 @@ struct FmtF32 {
         if (__uint_as_float(w4.x) == value) pos = 0;
         return pos;
     }
+    static __device__ __forceinline__ void mask_unit(uint4 &w4, int lo, int hi)
+    {
+        const uint32_t m = 0xe9045951u;   // -1e25
+        if (0 < lo || 0 >= hi) w4.x = m;
+        if (1 < lo || 1 >= hi) w4.y = m;
+        if (2 < lo || 2 >= hi) w4.z = m;
+        if (3 < lo || 3 >= hi) w4.w = m;
+    }
+};
+
+// Which logits of unit `ui` of a shifted row belong to the row: [lo, hi).
+struct RowEdges {
+    int32_t head, span, units;   // span = head + V
+    __device__ __forceinline__ bool touches(int32_t ui) const { return ui == 0 || ui == units - 1; }
+    template <typename Fmt>
+    __device__ __forceinline__ void mask(uint4 &w, int32_t ui) const
+    {
+        Fmt::mask_unit(w, ui == 0 ? head : 0, min(Fmt::EPU, span - ui * Fmt::EPU));
+    }
 };
 
 // One tile out of shared memory.  `nu` = units of this lane that exist (UNROLL unless MASKED);
-// refill() is called once every value of the stage sits in registers.
+// MASKED tiles of a shifted row (`edges` != nullptr) also blank the logits of the row's first and last unit that
+// belong to its neighbours.  refill() is called once every value of the stage sits in registers.
 template <bool MASKED, bool REV, typename Fmt, typename Refill>
 __device__ __forceinline__ void pipe_tile(const uint4 *sa, const uint4 *sb, int32_t u, int nu, RowAcc<REV> &acc,
-                                          float s, Refill refill)
+                                          float s, Refill refill, const RowEdges *edges = nullptr)
 {
     const int lane = threadIdx.x & 31;
     uint4 A[UNROLL], B[UNROLL];
@@ -320,6 +375,15 @@ __device__ __forceinline__ void pipe_tile(const uint4 *sa, const uint4 *sb, int3
     for (int j = 0; j < UNROLL; ++j) A[j] = (!MASKED || j < nu) ? sa[j * 32 + lane] : Fmt::none();
 #pragma unroll
     for (int j = 0; j < UNROLL; ++j) B[j] = (!MASKED || j < nu) ? sb[j * 32 + lane] : Fmt::none();
+    if (MASKED && edges) {
+#pragma unroll
+        for (int j = 0; j < UNROLL; ++j) {
+            if (j < nu && edges->touches(u + j * 32)) {
+                edges->template mask<Fmt>(A[j], u + j * 32);
+                edges->template mask<Fmt>(B[j], u + j * 32);
+            }
+        }
+    }
 
     const float tmax_a = Fmt::tile_max(A), tmax_b = Fmt::tile_max(B);
     acc.guard(tmax_a, tmax_b, s);
@@ -375,9 +439,10 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
     auto issue = [&](int st) -> int32_t {
         const int32_t n = min(TILE_UNITS, P.u1 - P.u);
         // the tile lies inside its row, the row inside the tensors, the stage inside the warp's ring
-        if (lane == 0 && PPOW_CHECK(n > 0 && P.u >= 0 && P.u + n <= job.units_per_row && st >= 0 && st < PIPE_STAGES &&
-                                        P.pa + P.u + n <= reinterpret_cast<const uint4 *>(job.target) +
-                                                              (size_t)job.N * job.K * job.units_per_row,
+        if (lane == 0 && PPOW_CHECK(n > 0 && P.u >= 0 && P.u + n <= P.units && st >= 0 && st < PIPE_STAGES &&
+                                        reinterpret_cast<uintptr_t>(P.pa + P.u + n) <=
+                                            ((reinterpret_cast<uintptr_t>(job.target) +
+                                              (size_t)job.N * job.K * (size_t)job.row_bytes + 15u) & ~(uintptr_t)15),
                                     101, &job.header->error_flags)) {
             const uint32_t bar = bars_addr + 8 * st, dst = stages_addr + st * 2 * TILE_BYTES;
             mbar_arrive_expect_tx(bar, 2u * (uint32_t)n * 16u);
@@ -442,10 +507,12 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
             __syncwarp();
             produce(st);
         };
-        if (n == TILE_UNITS)
+        const RowEdges edges = {C.head, C.head + job.V, C.units};
+        if (n == TILE_UNITS && (!job.shifted || (C.u > 0 && C.u + n < C.units)))
             pipe_tile<false, REV, Fmt>(sa, sb, C.u + lane, UNROLL, acc, job.s, refill);
         else
-            pipe_tile<true, REV, Fmt>(sa, sb, C.u + lane, min(UNROLL, (n - lane + 31) / 32), acc, job.s, refill);
+            pipe_tile<true, REV, Fmt>(sa, sb, C.u + lane, min(UNROLL, (n - lane + 31) / 32), acc, job.s, refill,
+                                      job.shifted ? &edges : nullptr);
         C.u += n;
 
         if (C.u >= C.u1) {   // end of the item: warp reduction, argmax index, one partial
@@ -457,11 +524,12 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
             const float item_max = warp_max(my_max);
             const bool holder = my_max == item_max;
             const int32_t bu = acc.best >> 3, bn = acc.best & 7;
+            const RowEdges done_edges = {C.head, C.head + job.V, C.units};
             uint4 cand[UNROLL];
 #pragma unroll
             for (int j = 0; j < UNROLL; ++j)
                 if (holder && j < bn &&
-                    PPOW_CHECK(bu >= 0 && bu + j * 32 < job.units_per_row, 102, &job.header->error_flags))
+                    PPOW_CHECK(bu >= 0 && bu + j * 32 < C.units, 102, &job.header->error_flags))
                     cand[j] = __ldcs(C.pa + bu + j * 32);
                 else
                     cand[j] = Fmt::none();
@@ -478,8 +546,9 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
 #pragma unroll
                 for (int j = 0; j < UNROLL; ++j) {
                     if (j < bn && arg == INT32_MAX) {
+                        if (job.shifted && done_edges.touches(bu + j * 32)) done_edges.template mask<Fmt>(cand[j], bu + j * 32);
                         const int pos = Fmt::first_equal(cand[j], my_max);
-                        if (pos >= 0) arg = (bu + j * 32) * Fmt::EPU + pos;
+                        if (pos >= 0) arg = (bu + j * 32) * Fmt::EPU + pos - done_edges.head;
                     }
                 }
             }
@@ -1018,12 +1087,17 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return PPOW_ERR_CUDA;
 
-    // the bulk-copy kernel needs rows of whole, 16-byte aligned units; everything else takes the scalar kernel
+    // The bulk-copy kernel reads 16-byte aligned units.  Rows of whole aligned units are the plain case; rows that
+    // start inside a unit (V not a multiple of the logits per unit, or a base pointer off a 16-byte boundary) are
+    // read from the aligned address below their start with their first and last unit masked, which needs both
+    // tensors at the same offset within a unit.  Tensors at different offsets take the scalar kernel.
     const int epu = params->dtype == PPOW_F32 ? FmtF32::EPU : FmtBf16::EPU;   // 8 logits per unit for both 16-bit types
-    const bool vec_ok = (params->V % epu == 0) && ((uintptr_t)draft_logits % 16 == 0) &&
-                        ((uintptr_t)target_logits % 16 == 0);
+    const bool vec_ok = ((uintptr_t)draft_logits % 16) == ((uintptr_t)target_logits % 16);
+    rj.shifted = (params->V % epu != 0) || ((uintptr_t)target_logits % 16 != 0);
     rj.units_per_row = params->V / epu;
     rj.tile_logits = TILE_UNITS * epu;
+    rj.es_shift = params->dtype == PPOW_F32 ? 2 : 1;
+    rj.row_bytes = (int64_t)params->V * (int64_t)esize;
     // one warp per work item in every row kernel: a grid that fills the GPU, or fewer CTAs when there is little work.
     // The kernels that also accumulate the sum for KL(Q||P) run only when that output is asked for.
     const void *kernel;

@@ -105,9 +105,12 @@ def _both_modes(x, c=0.05, temperature=1.0, eta=1.0, eps=0.5, ref_logp=None):
     # the same kinds of shape just past that limit reach the bulk-copy and the scalar kernels
     (5, 1, 2056, torch.bfloat16),       # bulk-copy kernel: two tiles and one unit
     (3, 32, 2064, torch.bfloat16),      # bulk-copy kernel, largest K
-    (7, 3, 5001, torch.bfloat16),       # odd V: scalar kernel, rows not 16-byte aligned
+    (7, 3, 5001, torch.bfloat16),       # odd V: rows start inside 16-byte units (bulk-copy kernel, first and last unit masked)
     (7, 3, 3001, torch.float32),
     (7, 3, 5001, torch.float16),
+    (5, 4, 50257, torch.bfloat16),      # a real odd vocabulary size: several items per row, every row at another offset
+    (3, 2, 128 * 8 * 3 + 1, torch.bfloat16),   # one logit more than three whole tiles: the last item gets an extra unit
+    (3, 2, 128 * 4 * 2 - 1, torch.float32),
     (2, 3, 1028, torch.float32),        # f32 bulk-copy kernel: two tiles and one unit
     (131, 4, 1000, torch.float32),      # one-launch kernel at its size limit (4 MiB of logits)
     (132, 4, 1000, torch.float32),      # the same rows just past the limit: bulk-copy kernel, one short item per row
@@ -133,15 +136,23 @@ def test_ragged_lengths_including_empty_windows():
         assert float(gpu[name][:3].float().abs().sum()) == 0.0     # empty windows: all outputs 0
 
 
-@pytest.mark.parametrize("V", [512, 4096])                       # one-launch kernel / scalar row kernel
-def test_unaligned_base_pointer_takes_scalar_path(V):
+@pytest.mark.parametrize("V,off_t,off_d", [
+    (512, 1, 1),        # one-launch kernel
+    (4096, 1, 1),       # both tensors one logit off a 16-byte boundary: bulk-copy kernel on shifted rows
+    (4096, 5, 5),
+    (4099, 0, 0),       # aligned base, odd V: every row starts at another offset
+    (4099, 3, 3),
+    (4096, 1, 3),       # tensors at different offsets within a unit: scalar row kernel
+    (4099, 0, 2),
+])
+def test_unaligned_rows_and_base_pointers(V, off_t, off_d):
     N, K = 3, 2
-    x = _random_inputs(N, K, V, torch.bfloat16, seed=6)
-    for key in ("target_logits", "draft_logits"):
-        flat = torch.empty(N * K * V + 1, dtype=torch.bfloat16, device=DEV)
-        flat[1:].copy_(x[key].flatten())
-        x[key] = flat[1:].view(N, K, V)                            # 2-byte aligned only
-        assert x[key].data_ptr() % 16 != 0
+    x = _random_inputs(N, K, V, torch.bfloat16, seed=6 + V + off_t)
+    for key, off in (("target_logits", off_t), ("draft_logits", off_d)):
+        flat = torch.full((N * K * V + 16,), 9000.0, dtype=torch.bfloat16, device=DEV)   # huge values around the tensor:
+        flat[off:off + N * K * V].copy_(x[key].flatten())                                # they must never be scored
+        x[key] = flat[off:off + N * K * V].view(N, K, V)
+        assert x[key].data_ptr() % 16 == (2 * off) % 16
     _both_modes(x)
 
 
@@ -194,6 +205,25 @@ def test_argmax_ties_take_lowest_index():
           "uniforms": torch.zeros((1, 1), device=DEV), "valid_len": None}
     gz, rz = _both_modes(xz)
     assert int(gz["target_argmax"][0, 0]) == 9 == int(rz["target_argmax"][0, 0])
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16, torch.float32])
+def test_argmax_ties_at_the_first_and_last_logit_of_rows_that_start_inside_a_unit(dtype):
+    # odd V: row r starts r * V logits into the tensor, at a different offset within a 16-byte unit each time; the
+    # maximum sits at the row's very first and very last logit (and once in the middle), next to the neighbours' data
+    N, K, V = 3, 3, 4099
+    x = _random_inputs(N, K, V, dtype, seed=23)
+    t = x["target_logits"]
+    top = t.float().amax(dim=(0, 1, 2)) + 1.0                       # one value above every row's maximum
+    t[:, :, V - 1] = top.to(dtype)
+    t[:, 1:, 2000] = top.to(dtype)
+    t[:, 2, 0] = top.to(dtype)
+    gpu, ref = _both_modes(x)
+    want = torch.tensor([V - 1, 2000, 0], device=DEV, dtype=torch.int32).expand(N, K)
+    assert torch.equal(gpu["target_argmax"], want)
+    x["draft_logits"] = x["target_logits"].clone()                   # and identical tensors still give exactly zero
+    g = run_gpu(x, "stochastic", 0.04)
+    assert float(g["kl"].abs().max()) == 0.0 and bool((g["accepted_len"] == K).all())
 
 
 def test_identical_logits_zero_divergence_full_acceptance():
