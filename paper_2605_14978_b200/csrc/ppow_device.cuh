@@ -191,6 +191,20 @@ struct RowAcc {
 };
 
 // ---- storage formats: one 16-byte unit of logits, and one logit at a time ---------------------------
+// mask_unit: the logits of a unit outside [lo, hi) do not belong to the row being read (a row that starts or
+// ends inside a unit); they are replaced by a finite, hugely negative value (-1e25, -65504 in binary16): its
+// term 2^x is 0 and 0 * x stays 0, which -inf would not.
+
+__device__ __forceinline__ void mask_halves(uint4 &w4, int lo, int hi, uint32_t bits)
+{
+    uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        if (2 * q < lo || 2 * q >= hi) w[q] = (w[q] & 0xffff0000u) | bits;
+        if (2 * q + 1 < lo || 2 * q + 1 >= hi) w[q] = (w[q] & 0x0000ffffu) | (bits << 16);
+    }
+    w4 = make_uint4(w[0], w[1], w[2], w[3]);
+}
 
 struct UnitBf16 {
     static constexpr int EPU = 8;   // logits per unit
@@ -205,6 +219,7 @@ struct UnitBf16 {
         f[0] = bf16_lo(w.x); f[1] = bf16_hi(w.x); f[2] = bf16_lo(w.y); f[3] = bf16_hi(w.y);
         f[4] = bf16_lo(w.z); f[5] = bf16_hi(w.z); f[6] = bf16_lo(w.w); f[7] = bf16_hi(w.w);
     }
+    static __device__ __forceinline__ void mask_unit(uint4 &w, int lo, int hi) { mask_halves(w, lo, hi, 0xe904u); }
 };
 
 struct UnitF16 {
@@ -222,6 +237,7 @@ struct UnitF16 {
         const float2 c = __half22float2(h2(w.z)), d = __half22float2(h2(w.w));
         f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y; f[4] = c.x; f[5] = c.y; f[6] = d.x; f[7] = d.y;
     }
+    static __device__ __forceinline__ void mask_unit(uint4 &w, int lo, int hi) { mask_halves(w, lo, hi, 0xfbffu); }
 };
 
 struct UnitF32 {
@@ -234,6 +250,43 @@ struct UnitF32 {
     static __device__ __forceinline__ void unpack(const uint4 &w, float (&f)[4])
     {
         f[0] = __uint_as_float(w.x); f[1] = __uint_as_float(w.y); f[2] = __uint_as_float(w.z); f[3] = __uint_as_float(w.w);
+    }
+    static __device__ __forceinline__ void mask_unit(uint4 &w, int lo, int hi)
+    {
+        const uint32_t m = 0xe9045951u;   // -1e25
+        if (0 < lo || 0 >= hi) w.x = m;
+        if (1 < lo || 1 >= hi) w.y = m;
+        if (2 < lo || 2 >= hi) w.z = m;
+        if (3 < lo || 3 >= hi) w.w = m;
+    }
+};
+
+// A row of V logits that may start inside a 16-byte unit: where its units begin, how many it spans, and which
+// logits of unit `ui` belong to it.
+template <typename Unit>
+struct RowSpan {
+    const uint4 *base;     // aligned address of the unit that holds the row's first logit
+    int32_t head, span, units;   // logits of unit 0 before the row; head + V; units the row touches
+    __device__ __forceinline__ RowSpan(const void *tensor, size_t row, int32_t V)
+    {
+        constexpr int ES = 16 / Unit::EPU;
+        const uintptr_t a = reinterpret_cast<uintptr_t>(tensor) + row * (size_t)V * ES;
+        base = reinterpret_cast<const uint4 *>(a & ~(uintptr_t)15);
+        head = (int32_t)((a & 15u) / ES);
+        span = head + V;
+        units = (span + Unit::EPU - 1) / Unit::EPU;
+    }
+    __device__ __forceinline__ bool touches(int32_t ui) const { return ui == 0 || ui == units - 1; }
+    __device__ __forceinline__ void mask(uint4 &w, int32_t ui) const
+    {
+        Unit::mask_unit(w, ui == 0 ? head : 0, min(Unit::EPU, span - ui * Unit::EPU));
+    }
+    // unit ui of the row with the neighbours' logits blanked
+    __device__ __forceinline__ uint4 load(const uint4 *p, int32_t ui) const
+    {
+        uint4 w = __ldcs(p + ui);
+        if (touches(ui)) mask(w, ui);
+        return w;
     }
 };
 

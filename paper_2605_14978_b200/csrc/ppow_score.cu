@@ -190,6 +190,7 @@ struct ItemCursor {
     const uint4 *pa, *pb;   // first unit of the row in each tensor (16-byte aligned)
 };
 
+template <bool SHIFTED>
 __device__ __forceinline__ void open_item(const RowJob &job, ItemCursor &c, uint32_t item)
 {
     c.item = item;
@@ -200,7 +201,7 @@ __device__ __forceinline__ void open_item(const RowJob &job, ItemCursor &c, uint
     uint32_t row;
     int32_t t0, t1;
     locate_item(job.plan, item, row, t0, t1);
-    if (!job.shifted) {
+    if (!SHIFTED) {
         c.units = job.units_per_row;
         c.pa = reinterpret_cast<const uint4 *>(job.target) + (size_t)row * c.units;
         c.pb = reinterpret_cast<const uint4 *>(job.draft) + (size_t)row * c.units;
@@ -219,8 +220,6 @@ __device__ __forceinline__ void open_item(const RowJob &job, ItemCursor &c, uint
     c.u = t0 * TILE_UNITS;
     c.u1 = (t1 == job.plan.tiles) ? c.units : t1 * TILE_UNITS;   // the last item of a row takes what is left of it
 }
-
-__device__ __forceinline__ void mask_halves(uint4 &w4, int lo, int hi, uint32_t bits);
 
 // Storage formats of the bulk-copy kernel: how a 16-byte unit of logits is read.
 struct FmtBf16 {
@@ -258,21 +257,8 @@ struct FmtBf16 {
         }
         return pos;
     }
-    // logits outside [lo, hi) of the unit do not belong to the row: replaced by a finite, hugely negative value
-    // (-1e25: its term 2^x is 0 and 0 * x stays 0, which -inf would not)
-    static __device__ __forceinline__ void mask_unit(uint4 &w4, int lo, int hi) { mask_halves(w4, lo, hi, 0xe904u); }
+    static __device__ __forceinline__ void mask_unit(uint4 &w4, int lo, int hi) { UnitBf16::mask_unit(w4, lo, hi); }
 };
-
-__device__ __forceinline__ void mask_halves(uint4 &w4, int lo, int hi, uint32_t bits)
-{
-    uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        if (2 * q < lo || 2 * q >= hi) w[q] = (w[q] & 0xffff0000u) | bits;
-        if (2 * q + 1 < lo || 2 * q + 1 >= hi) w[q] = (w[q] & 0x0000ffffu) | (bits << 16);
-    }
-    w4 = make_uint4(w[0], w[1], w[2], w[3]);
-}
 
 struct FmtF16 {
     static constexpr int EPU = 8;
@@ -308,7 +294,7 @@ struct FmtF16 {
         }
         return pos;
     }
-    static __device__ __forceinline__ void mask_unit(uint4 &w4, int lo, int hi) { mask_halves(w4, lo, hi, 0xfbffu); }   // -65504
+    static __device__ __forceinline__ void mask_unit(uint4 &w4, int lo, int hi) { UnitF16::mask_unit(w4, lo, hi); }
 };
 
 struct FmtF32 {
@@ -341,14 +327,7 @@ struct FmtF32 {
         if (__uint_as_float(w4.x) == value) pos = 0;
         return pos;
     }
-    static __device__ __forceinline__ void mask_unit(uint4 &w4, int lo, int hi)
-    {
-        const uint32_t m = 0xe9045951u;   // -1e25
-        if (0 < lo || 0 >= hi) w4.x = m;
-        if (1 < lo || 1 >= hi) w4.y = m;
-        if (2 < lo || 2 >= hi) w4.z = m;
-        if (3 < lo || 3 >= hi) w4.w = m;
-    }
+    static __device__ __forceinline__ void mask_unit(uint4 &w4, int lo, int hi) { UnitF32::mask_unit(w4, lo, hi); }
 };
 
 // Which logits of unit `ui` of a shifted row belong to the row: [lo, hi).
@@ -400,7 +379,8 @@ __device__ __forceinline__ void pipe_tile(const uint4 *sa, const uint4 *sb, int3
     acc.flush();
 }
 
-template <bool REV, typename Fmt>
+// SHIFTED: rows that start inside a 16-byte unit (instances of their own, so that the plain case pays nothing for it).
+template <bool REV, typename Fmt, bool SHIFTED>
 __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pipe_kernel(const RowJob job)
 {
     extern __shared__ __align__(128) unsigned char pipe_smem[];
@@ -431,7 +411,7 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
     uint32_t upcoming = 0;                  // (lane 0) id fetched ahead for the item after P's
     const uint32_t first = first_item(job, blockIdx.x * PIPE_WARPS + warp, workers, lane);
     if (lane == 0) item_ring[warp][0] = first;
-    open_item(job, P, first);
+    open_item<SHIFTED>(job, P, first);
     C = P;
     produced = consumed = 1;
 
@@ -462,7 +442,7 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
                 if (nx < job.total_items) upcoming = fetch_item(job, workers);
             }
             ++produced;
-            open_item(job, P, nx);
+            open_item<SHIFTED>(job, P, nx);
         }
     };
     auto produce = [&](int st) {
@@ -508,11 +488,11 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
             produce(st);
         };
         const RowEdges edges = {C.head, C.head + job.V, C.units};
-        if (n == TILE_UNITS && (!job.shifted || (C.u > 0 && C.u + n < C.units)))
+        if (n == TILE_UNITS && (!SHIFTED || (C.u > 0 && C.u + n < C.units)))
             pipe_tile<false, REV, Fmt>(sa, sb, C.u + lane, UNROLL, acc, job.s, refill);
         else
             pipe_tile<true, REV, Fmt>(sa, sb, C.u + lane, min(UNROLL, (n - lane + 31) / 32), acc, job.s, refill,
-                                      job.shifted ? &edges : nullptr);
+                                      SHIFTED ? &edges : nullptr);
         C.u += n;
 
         if (C.u >= C.u1) {   // end of the item: warp reduction, argmax index, one partial
@@ -540,13 +520,13 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
             __syncwarp();
             const uint32_t nx = item_ring[warp][consumed % ITEM_RING];
             ++consumed;
-            open_item(job, C, nx);
+            open_item<SHIFTED>(job, C, nx);
             int32_t arg = INT32_MAX;
             if (holder) {
 #pragma unroll
                 for (int j = 0; j < UNROLL; ++j) {
                     if (j < bn && arg == INT32_MAX) {
-                        if (job.shifted && done_edges.touches(bu + j * 32)) done_edges.template mask<Fmt>(cand[j], bu + j * 32);
+                        if (SHIFTED && done_edges.touches(bu + j * 32)) done_edges.template mask<Fmt>(cand[j], bu + j * 32);
                         const int pos = Fmt::first_equal(cand[j], my_max);
                         if (pos >= 0) arg = (bu + j * 32) * Fmt::EPU + pos - done_edges.head;
                     }
@@ -981,7 +961,7 @@ static bool takes_small_path(const ppow_params *p)
 // and remembered: the dynamic shared memory opt-in, the occupancy query and the SM count are host calls
 // of several microseconds each, as much as a small problem's whole launch.  (Launch limits of a device are
 // the only thing the library remembers between calls; concurrent first calls store the same value.)
-constexpr int CACHE_DEVICES = 64, CACHE_KERNELS = 12;
+constexpr int CACHE_DEVICES = 64, CACHE_KERNELS = 18;
 static std::atomic<int> g_resident_ctas[CACHE_DEVICES][CACHE_KERNELS];
 
 static int resident_ctas(int dev, int kernel_index, const void *kernel, int threads, size_t dyn_smem)
@@ -1104,12 +1084,11 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
     int threads = ROW_THREADS;
     size_t dyn_smem = 0;
     if (vec_ok) {
-        if (params->dtype == PPOW_BF16)
-            kernel = rev ? (const void *)row_reduce_pipe_kernel<true, FmtBf16> : (const void *)row_reduce_pipe_kernel<false, FmtBf16>;
-        else if (params->dtype == PPOW_F16)
-            kernel = rev ? (const void *)row_reduce_pipe_kernel<true, FmtF16> : (const void *)row_reduce_pipe_kernel<false, FmtF16>;
-        else
-            kernel = rev ? (const void *)row_reduce_pipe_kernel<true, FmtF32> : (const void *)row_reduce_pipe_kernel<false, FmtF32>;
+        const bool sh = rj.shifted != 0;
+#define PPOW_PIPE(FMT) (rev ? (sh ? (const void *)row_reduce_pipe_kernel<true, FMT, true> : (const void *)row_reduce_pipe_kernel<true, FMT, false>) \
+                            : (sh ? (const void *)row_reduce_pipe_kernel<false, FMT, true> : (const void *)row_reduce_pipe_kernel<false, FMT, false>))
+        kernel = params->dtype == PPOW_BF16 ? PPOW_PIPE(FmtBf16) : params->dtype == PPOW_F16 ? PPOW_PIPE(FmtF16) : PPOW_PIPE(FmtF32);
+#undef PPOW_PIPE
         threads = PIPE_WARPS * 32;
         dyn_smem = PIPE_SMEM_BYTES;
     } else if (params->dtype == PPOW_BF16) {
@@ -1122,7 +1101,7 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
         kernel = rev ? (const void *)row_reduce_generic_kernel<float, true>
                      : (const void *)row_reduce_generic_kernel<float, false>;
     }
-    const int kernel_index = (vec_ok ? 6 : 0) + 2 * params->dtype + (rev ? 1 : 0);
+    const int kernel_index = (vec_ok ? (rj.shifted ? 12 : 6) : 0) + 2 * params->dtype + (rev ? 1 : 0);
     const int resident = resident_ctas(dev, kernel_index, kernel, threads, dyn_smem);
     if (resident < 1) return PPOW_ERR_CUDA;
     const unsigned warps_per_cta = (unsigned)threads / 32;

@@ -146,7 +146,7 @@ __global__ void __launch_bounds__(ACC_THREADS) expected_acceptance_vec_kernel(co
                                                                               const int32_t *__restrict__ valid_len,
                                                                               const float *__restrict__ lse_p,
                                                                               const float *__restrict__ lse_q, int32_t K,
-                                                                              int32_t units, float s,
+                                                                              int32_t V, float s,
                                                                               float *__restrict__ out)
 {
     __shared__ double warp_part[ACC_THREADS / 32];
@@ -159,9 +159,13 @@ __global__ void __launch_bounds__(ACC_THREADS) expected_acceptance_vec_kernel(co
     }
     // P(v) = 2^(a*s - la), Q(v) = 2^(b*s - lb) with the normalisers converted to log2 units
     const float la = lse_p[row] * 1.4426950408889634f, lb = lse_q[row] * 1.4426950408889634f;
-    const uint4 *pa = target + row * (size_t)units, *pb = draft + row * (size_t)units;
+    // rows may start inside a 16-byte unit (odd V, offset base): both tensors at the same offset; the logits of
+    // the first and last unit that belong to the neighbouring rows are blanked (they then add min(0, 0))
+    const RowSpan<Unit> ra(target, row, V), rb(draft, row, V);
+    const uint4 *pa = ra.base, *pb = rb.base;
+    const int32_t units = ra.units;
     float acc0 = 0.0f, acc1 = 0.0f;
-    if (!PPOW_CHECK(row < (size_t)gridDim.x && k < K, 402, nullptr)) return;
+    if (!PPOW_CHECK(row < (size_t)gridDim.x && k < K && ra.head == rb.head, 402, nullptr)) return;
     auto add_unit = [&](const uint4 &A, const uint4 &B) {
         float fa[Unit::EPU], fb[Unit::EPU];
         Unit::unpack(A, fa);
@@ -174,12 +178,12 @@ __global__ void __launch_bounds__(ACC_THREADS) expected_acceptance_vec_kernel(co
     };
     int32_t u = tid;
     for (; u + ACC_THREADS < units; u += 2 * ACC_THREADS) {
-        const uint4 A0 = __ldcs(pa + u), B0 = __ldcs(pb + u);
-        const uint4 A1 = __ldcs(pa + u + ACC_THREADS), B1 = __ldcs(pb + u + ACC_THREADS);
+        const uint4 A0 = ra.load(pa, u), B0 = rb.load(pb, u);
+        const uint4 A1 = ra.load(pa, u + ACC_THREADS), B1 = rb.load(pb, u + ACC_THREADS);
         add_unit(A0, B0);
         add_unit(A1, B1);
     }
-    if (u < units) add_unit(__ldcs(pa + u), __ldcs(pb + u));
+    if (u < units) add_unit(ra.load(pa, u), rb.load(pb, u));
     const double w = warp_sum_f64((double)acc0 + (double)acc1);
     if ((tid & 31) == 0) warp_part[tid >> 5] = w;
     __syncthreads();
@@ -293,7 +297,7 @@ __device__ __forceinline__ void lse_block_finish(const LseAcc &acc, float s, flo
 template <typename Unit>
 __global__ void __launch_bounds__(REF_THREADS) reference_logprob_vec_kernel(const uint4 *__restrict__ ref,
                                                                             const int32_t *__restrict__ valid_len,
-                                                                            int32_t K, int32_t units, float s,
+                                                                            int32_t K, int32_t V, float s,
                                                                             float *__restrict__ row_logp)
 {
     const size_t row = blockIdx.x;
@@ -305,7 +309,9 @@ __global__ void __launch_bounds__(REF_THREADS) reference_logprob_vec_kernel(cons
     }
     LseAcc acc;
     acc.reset();
-    const uint4 *p = ref + row * (size_t)units;
+    const RowSpan<Unit> rs(ref, row, V);   // the row may start inside a 16-byte unit: first and last unit are blanked
+    const uint4 *p = rs.base;
+    const int32_t units = rs.units;
     auto add_unit = [&](const uint4 &w) {
         float f[Unit::EPU];
         Unit::unpack(w, f);
@@ -316,8 +322,8 @@ __global__ void __launch_bounds__(REF_THREADS) reference_logprob_vec_kernel(cons
     // the memory system short of requests), one reference check and one fold per round
     int32_t u = tid;
     for (; u + 3 * REF_THREADS < units; u += 4 * REF_THREADS) {
-        const uint4 w0 = __ldcs(p + u), w1 = __ldcs(p + u + REF_THREADS);
-        const uint4 w2 = __ldcs(p + u + 2 * REF_THREADS), w3 = __ldcs(p + u + 3 * REF_THREADS);
+        const uint4 w0 = rs.load(p, u), w1 = rs.load(p, u + REF_THREADS);
+        const uint4 w2 = rs.load(p, u + 2 * REF_THREADS), w3 = rs.load(p, u + 3 * REF_THREADS);
         acc.guard(fmaxf(fmaxf(Unit::unit_max(w0), Unit::unit_max(w1)), fmaxf(Unit::unit_max(w2), Unit::unit_max(w3))), s);
         add_unit(w0);
         add_unit(w1);
@@ -327,34 +333,9 @@ __global__ void __launch_bounds__(REF_THREADS) reference_logprob_vec_kernel(cons
         acc.fold();
     }
     for (; u < units; u += REF_THREADS) {
-        const uint4 w0 = __ldcs(p + u);
+        const uint4 w0 = rs.load(p, u);
         acc.guard(Unit::unit_max(w0), s);
         add_unit(w0);
-        acc.fold();
-    }
-    lse_block_finish(acc, s, row_logp + row);
-}
-
-template <typename T>
-__global__ void __launch_bounds__(REF_THREADS) reference_logprob_scalar_kernel(const T *__restrict__ ref,
-                                                                               const int32_t *__restrict__ valid_len,
-                                                                               int32_t K, int32_t V, float s,
-                                                                               float *__restrict__ row_logp)
-{
-    const size_t row = blockIdx.x;
-    const int32_t n = (int32_t)(row / (size_t)K), k = (int32_t)(row % (size_t)K);
-    const int tid = threadIdx.x;
-    if (valid_len && k >= valid_len[n]) {
-        if (tid == 0) row_logp[row] = 0.0f;
-        return;
-    }
-    LseAcc acc;
-    acc.reset();
-    const T *p = ref + row * (size_t)V;
-    for (int32_t i = tid; i < V; i += REF_THREADS) {
-        const float v = load_logit<T>(p, i);
-        acc.guard(v, s);
-        acc.add(v, s);
         acc.fold();
     }
     lse_block_finish(acc, s, row_logp + row);
@@ -441,14 +422,15 @@ extern "C" ppow_status ppow_expected_acceptance(const ppow_params *params,
     const float s = (float)(1.4426950408889634074 / (double)params->temperature);
     const int32_t K = params->K, V = params->V;
     const int epu = params->dtype == PPOW_F32 ? 4 : 8;
-    const bool vec = V % epu == 0 && (uintptr_t)draft_logits % 16 == 0 && (uintptr_t)target_logits % 16 == 0;
+    (void)epu;
+    const bool vec = (uintptr_t)draft_logits % 16 == (uintptr_t)target_logits % 16;   // same offset within a 16-byte unit
     const uint4 *ta = (const uint4 *)target_logits, *da = (const uint4 *)draft_logits;
     if (vec && params->dtype == PPOW_BF16)
-        expected_acceptance_vec_kernel<UnitBf16><<<rows, ACC_THREADS, 0, stream>>>(ta, da, valid_len, lse_p, lse_q, K, V / epu, s, expected_accept);
+        expected_acceptance_vec_kernel<UnitBf16><<<rows, ACC_THREADS, 0, stream>>>(ta, da, valid_len, lse_p, lse_q, K, V, s, expected_accept);
     else if (vec && params->dtype == PPOW_F16)
-        expected_acceptance_vec_kernel<UnitF16><<<rows, ACC_THREADS, 0, stream>>>(ta, da, valid_len, lse_p, lse_q, K, V / epu, s, expected_accept);
+        expected_acceptance_vec_kernel<UnitF16><<<rows, ACC_THREADS, 0, stream>>>(ta, da, valid_len, lse_p, lse_q, K, V, s, expected_accept);
     else if (vec)
-        expected_acceptance_vec_kernel<UnitF32><<<rows, ACC_THREADS, 0, stream>>>(ta, da, valid_len, lse_p, lse_q, K, V / epu, s, expected_accept);
+        expected_acceptance_vec_kernel<UnitF32><<<rows, ACC_THREADS, 0, stream>>>(ta, da, valid_len, lse_p, lse_q, K, V, s, expected_accept);
     else if (params->dtype == PPOW_F32)
         expected_acceptance_scalar_kernel<float><<<rows, ACC_THREADS, 0, stream>>>(
             (const float *)target_logits, (const float *)draft_logits, valid_len, lse_p, lse_q, K, V, s, expected_accept);
@@ -477,21 +459,14 @@ extern "C" ppow_status ppow_reference_logprob(const ppow_params *params, const v
     const float s = (float)(1.4426950408889634074 / (double)params->temperature);
     const unsigned rows = (unsigned)((size_t)params->N * params->K);
     const int32_t K = params->K, V = params->V;
-    const int epu = params->dtype == PPOW_F32 ? 4 : 8;
-    const bool vec = V % epu == 0 && (uintptr_t)ref_target_logits % 16 == 0;
+    // any V and any element-aligned base: rows that start inside a 16-byte unit are masked at their ends
     const uint4 *ra = (const uint4 *)ref_target_logits;
-    if (vec && params->dtype == PPOW_BF16)
-        reference_logprob_vec_kernel<UnitBf16><<<rows, REF_THREADS, 0, stream>>>(ra, valid_len, K, V / epu, s, row_logp);
-    else if (vec && params->dtype == PPOW_F16)
-        reference_logprob_vec_kernel<UnitF16><<<rows, REF_THREADS, 0, stream>>>(ra, valid_len, K, V / epu, s, row_logp);
-    else if (vec)
-        reference_logprob_vec_kernel<UnitF32><<<rows, REF_THREADS, 0, stream>>>(ra, valid_len, K, V / epu, s, row_logp);
-    else if (params->dtype == PPOW_F32)
-        reference_logprob_scalar_kernel<float><<<rows, REF_THREADS, 0, stream>>>((const float *)ref_target_logits, valid_len, K, V, s, row_logp);
+    if (params->dtype == PPOW_BF16)
+        reference_logprob_vec_kernel<UnitBf16><<<rows, REF_THREADS, 0, stream>>>(ra, valid_len, K, V, s, row_logp);
     else if (params->dtype == PPOW_F16)
-        reference_logprob_scalar_kernel<half_bits><<<rows, REF_THREADS, 0, stream>>>((const half_bits *)ref_target_logits, valid_len, K, V, s, row_logp);
+        reference_logprob_vec_kernel<UnitF16><<<rows, REF_THREADS, 0, stream>>>(ra, valid_len, K, V, s, row_logp);
     else
-        reference_logprob_scalar_kernel<uint16_t><<<rows, REF_THREADS, 0, stream>>>((const uint16_t *)ref_target_logits, valid_len, K, V, s, row_logp);
+        reference_logprob_vec_kernel<UnitF32><<<rows, REF_THREADS, 0, stream>>>(ra, valid_len, K, V, s, row_logp);
     if (cudaGetLastError() != cudaSuccess) return PPOW_ERR_CUDA;
     if (ref_logp) {
         reference_logprob_sum_kernel<<<(unsigned)((params->N + 127) / 128), 128, 0, stream>>>(row_logp, valid_len, params->N,

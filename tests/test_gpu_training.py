@@ -300,6 +300,33 @@ def test_expected_acceptance_scalar_path_and_identical_distributions():
     np.testing.assert_allclose(acc.cpu().numpy(), 1.0, atol=2e-5)    # min(P, P) sums to 1
 
 
+@pytest.mark.parametrize("V,off_t,off_d,dtype", [(4099, 0, 0, torch.bfloat16), (4096, 3, 3, torch.bfloat16),
+                                                 (4099, 1, 1, torch.float16), (2051, 1, 1, torch.float32),
+                                                 (4096, 1, 3, torch.bfloat16), (2051, 0, 2, torch.float32)])
+def test_expected_acceptance_and_reference_logprob_on_rows_that_start_inside_a_unit(V, off_t, off_d, dtype):
+    # odd V and base pointers off a 16-byte boundary: same offset -> vector kernels with the first and last unit of
+    # a row masked; different offsets -> the scalar expected-acceptance kernel.  Huge values surround the tensors.
+    N, K, T = 4, 3, 0.9
+    g = torch.Generator(device=DEV).manual_seed(V + off_t + 7 * off_d)
+    t = torch.randn((N, K, V), generator=g, device=DEV) * 2.0
+    d = t + 0.8 * torch.randn((N, K, V), generator=g, device=DEV)
+    x = {"draft_tokens": torch.randint(0, V, (N, K), generator=g, device=DEV, dtype=torch.int32), "uniforms": None,
+         "valid_len": None}
+    for key, val, off in (("target_logits", t, off_t), ("draft_logits", d, off_d)):
+        flat = torch.full((N * K * V + 16,), 9000.0, dtype=dtype, device=DEV)
+        flat[off:off + N * K * V].copy_(val.to(dtype).flatten())
+        x[key] = flat[off:off + N * K * V].view(N, K, V)
+    gpu = _score_with_training_outputs(x, "greedy", 0.05, T)
+    params = B.make_params(N, K, V, B.DTYPE_CODES[dtype], B.PPOW_GREEDY, 0.05, T)
+    acc = torch.empty((N, K), device=DEV)
+    B.ppow_expected_acceptance(params, x["draft_logits"], x["target_logits"], None, gpu["lse_p"], gpu["lse_q"], acc)
+    row_logp, ref_logp = torch.empty((N, K), device=DEV), torch.empty((N,), device=DEV)
+    B.ppow_reference_logprob(params, x["target_logits"], None, row_logp, ref_logp)
+    torch.cuda.synchronize()
+    _assert_close("expected_accept", acc.cpu().numpy(), _oracle_diag(x, T)["expected_accept"])
+    _assert_close("ref_logp", ref_logp.cpu().numpy(), oracle.reference_logprob(x["target_logits"].cpu(), temperature=T))
+
+
 # ------------------------------------------------------------------ reference-window log-probability (exact Delta)
 
 
