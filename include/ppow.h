@@ -100,7 +100,14 @@ size_t ppow_score_workspace_bytes(const ppow_params *params);
  * verification, proximity-gap and reward steps of Alg. 1).
  *
  *   draft_logits, target_logits  device, [N,K,V] of params->dtype (float32, bfloat16 or IEEE float16),
- *                                contiguous.  Both tensors are read from HBM exactly once.
+ *                                contiguous, aligned to their element size.  Both tensors are read from HBM
+ *                                exactly once, in aligned 16-byte units: when V is not a multiple of the logits
+ *                                per unit, or a base pointer is off a 16-byte boundary, the units that hold a
+ *                                row's first and last logit are read whole (the neighbours' logits in them are
+ *                                masked out), so up to 15 bytes before the first and after the last logit of a
+ *                                tensor are read too -- bytes of the same aligned 16-byte unit as valid data.
+ *                                Full speed needs both tensors at the same offset within a unit (any offset);
+ *                                otherwise a slower scalar kernel runs.
  *   draft_tokens                 device, [N,K] int32.  A token outside [0,V) is rejected, gets
  *                                logp_tok = logq_tok = -inf, and sets PPOW_FLAG_TOKEN_RANGE.
  *   uniforms                     device, [N,K] float32 in [0,1), drawn by the caller;

@@ -261,9 +261,9 @@ struct UnitF32 {
     }
 };
 
-// A row of V logits that may start inside a 16-byte unit: where its units begin, how many it spans, and which
-// logits of unit `ui` belong to it.
-template <typename Unit>
+// A row of V logits that may start inside a 16-byte unit (SHIFTED; otherwise rows are whole aligned units and
+// nothing is masked): where its units begin, how many it spans, and which logits of unit `ui` belong to it.
+template <typename Unit, bool SHIFTED>
 struct RowSpan {
     const uint4 *base;     // aligned address of the unit that holds the row's first logit
     int32_t head, span, units;   // logits of unit 0 before the row; head + V; units the row touches
@@ -272,7 +272,7 @@ struct RowSpan {
         constexpr int ES = 16 / Unit::EPU;
         const uintptr_t a = reinterpret_cast<uintptr_t>(tensor) + row * (size_t)V * ES;
         base = reinterpret_cast<const uint4 *>(a & ~(uintptr_t)15);
-        head = (int32_t)((a & 15u) / ES);
+        head = SHIFTED ? (int32_t)((a & 15u) / ES) : 0;
         span = head + V;
         units = (span + Unit::EPU - 1) / Unit::EPU;
     }
@@ -285,7 +285,7 @@ struct RowSpan {
     __device__ __forceinline__ uint4 load(const uint4 *p, int32_t ui) const
     {
         uint4 w = __ldcs(p + ui);
-        if (touches(ui)) mask(w, ui);
+        if (SHIFTED && touches(ui)) mask(w, ui);
         return w;
     }
 };

@@ -140,7 +140,7 @@ constexpr int ACC_THREADS = 256;
 
 // Rows of whole, 16-byte aligned units of any storage format: 16-byte streaming loads, two units of each
 // tensor in flight per thread.
-template <typename Unit>
+template <typename Unit, bool SHIFTED>
 __global__ void __launch_bounds__(ACC_THREADS) expected_acceptance_vec_kernel(const uint4 *__restrict__ target,
                                                                               const uint4 *__restrict__ draft,
                                                                               const int32_t *__restrict__ valid_len,
@@ -161,7 +161,7 @@ __global__ void __launch_bounds__(ACC_THREADS) expected_acceptance_vec_kernel(co
     const float la = lse_p[row] * 1.4426950408889634f, lb = lse_q[row] * 1.4426950408889634f;
     // rows may start inside a 16-byte unit (odd V, offset base): both tensors at the same offset; the logits of
     // the first and last unit that belong to the neighbouring rows are blanked (they then add min(0, 0))
-    const RowSpan<Unit> ra(target, row, V), rb(draft, row, V);
+    const RowSpan<Unit, SHIFTED> ra(target, row, V), rb(draft, row, V);
     const uint4 *pa = ra.base, *pb = rb.base;
     const int32_t units = ra.units;
     float acc0 = 0.0f, acc1 = 0.0f;
@@ -294,7 +294,7 @@ __device__ __forceinline__ void lse_block_finish(const LseAcc &acc, float s, flo
 
 // One CTA per (window, position) row from a plain grid; writes log max_v P(v) of the row.
 // Rows of whole, 16-byte aligned units of any storage format (one fold per 8 or 16 logits).
-template <typename Unit>
+template <typename Unit, bool SHIFTED>
 __global__ void __launch_bounds__(REF_THREADS) reference_logprob_vec_kernel(const uint4 *__restrict__ ref,
                                                                             const int32_t *__restrict__ valid_len,
                                                                             int32_t K, int32_t V, float s,
@@ -309,7 +309,7 @@ __global__ void __launch_bounds__(REF_THREADS) reference_logprob_vec_kernel(cons
     }
     LseAcc acc;
     acc.reset();
-    const RowSpan<Unit> rs(ref, row, V);   // the row may start inside a 16-byte unit: first and last unit are blanked
+    const RowSpan<Unit, SHIFTED> rs(ref, row, V);   // the row may start inside a 16-byte unit: first and last unit are blanked
     const uint4 *p = rs.base;
     const int32_t units = rs.units;
     auto add_unit = [&](const uint4 &w) {
@@ -422,15 +422,25 @@ extern "C" ppow_status ppow_expected_acceptance(const ppow_params *params,
     const float s = (float)(1.4426950408889634074 / (double)params->temperature);
     const int32_t K = params->K, V = params->V;
     const int epu = params->dtype == PPOW_F32 ? 4 : 8;
-    (void)epu;
     const bool vec = (uintptr_t)draft_logits % 16 == (uintptr_t)target_logits % 16;   // same offset within a 16-byte unit
     const uint4 *ta = (const uint4 *)target_logits, *da = (const uint4 *)draft_logits;
+    const bool shifted = V % epu != 0 || (uintptr_t)target_logits % 16 != 0;   // rows that start inside a unit
+#define PPOW_ACC(UNIT)                                                                                          \
+    do {                                                                                                        \
+        if (shifted)                                                                                            \
+            expected_acceptance_vec_kernel<UNIT, true><<<rows, ACC_THREADS, 0, stream>>>(ta, da, valid_len, lse_p, lse_q, K, \
+                                                                                          V, s, expected_accept); \
+        else                                                                                                    \
+            expected_acceptance_vec_kernel<UNIT, false><<<rows, ACC_THREADS, 0, stream>>>(ta, da, valid_len, lse_p, lse_q, K, \
+                                                                                           V, s, expected_accept); \
+    } while (0)
     if (vec && params->dtype == PPOW_BF16)
-        expected_acceptance_vec_kernel<UnitBf16><<<rows, ACC_THREADS, 0, stream>>>(ta, da, valid_len, lse_p, lse_q, K, V, s, expected_accept);
+        PPOW_ACC(UnitBf16);
     else if (vec && params->dtype == PPOW_F16)
-        expected_acceptance_vec_kernel<UnitF16><<<rows, ACC_THREADS, 0, stream>>>(ta, da, valid_len, lse_p, lse_q, K, V, s, expected_accept);
+        PPOW_ACC(UnitF16);
     else if (vec)
-        expected_acceptance_vec_kernel<UnitF32><<<rows, ACC_THREADS, 0, stream>>>(ta, da, valid_len, lse_p, lse_q, K, V, s, expected_accept);
+        PPOW_ACC(UnitF32);
+#undef PPOW_ACC
     else if (params->dtype == PPOW_F32)
         expected_acceptance_scalar_kernel<float><<<rows, ACC_THREADS, 0, stream>>>(
             (const float *)target_logits, (const float *)draft_logits, valid_len, lse_p, lse_q, K, V, s, expected_accept);
@@ -461,12 +471,21 @@ extern "C" ppow_status ppow_reference_logprob(const ppow_params *params, const v
     const int32_t K = params->K, V = params->V;
     // any V and any element-aligned base: rows that start inside a 16-byte unit are masked at their ends
     const uint4 *ra = (const uint4 *)ref_target_logits;
+    const bool shifted = V % (params->dtype == PPOW_F32 ? 4 : 8) != 0 || (uintptr_t)ref_target_logits % 16 != 0;
+#define PPOW_REF(UNIT)                                                                                                   \
+    do {                                                                                                                 \
+        if (shifted)                                                                                                     \
+            reference_logprob_vec_kernel<UNIT, true><<<rows, REF_THREADS, 0, stream>>>(ra, valid_len, K, V, s, row_logp); \
+        else                                                                                                             \
+            reference_logprob_vec_kernel<UNIT, false><<<rows, REF_THREADS, 0, stream>>>(ra, valid_len, K, V, s, row_logp); \
+    } while (0)
     if (params->dtype == PPOW_BF16)
-        reference_logprob_vec_kernel<UnitBf16><<<rows, REF_THREADS, 0, stream>>>(ra, valid_len, K, V, s, row_logp);
+        PPOW_REF(UnitBf16);
     else if (params->dtype == PPOW_F16)
-        reference_logprob_vec_kernel<UnitF16><<<rows, REF_THREADS, 0, stream>>>(ra, valid_len, K, V, s, row_logp);
+        PPOW_REF(UnitF16);
     else
-        reference_logprob_vec_kernel<UnitF32><<<rows, REF_THREADS, 0, stream>>>(ra, valid_len, K, V, s, row_logp);
+        PPOW_REF(UnitF32);
+#undef PPOW_REF
     if (cudaGetLastError() != cudaSuccess) return PPOW_ERR_CUDA;
     if (ref_logp) {
         reference_logprob_sum_kernel<<<(unsigned)((params->N + 127) / 128), 128, 0, stream>>>(row_logp, valid_len, params->N,
