@@ -346,11 +346,12 @@ ppow_status ppow_checked_failures(uint32_t *failures_host, uint32_t *first_site_
 
 /*
  * Timeline build (an addition of this library; the paper has no counterpart).  The build script can also
- * produce libppow_timeline.so (-DPPOW_TIMELINE), in which every warp of the bulk-copy row kernel records nine
+ * produce libppow_timeline.so (-DPPOW_TIMELINE), in which every warp of the bulk-copy row kernel records eleven
  * 64-bit words per launch: start, first data arrival and end (global timer, ns), items and tiles it processed,
- * its SM, cycles spent waiting for copies, cycles spent in item ends, and its total cycles.  This call
+ * its SM, cycles spent waiting for copies, cycles spent in item ends, its total cycles, and the item-end cycles
+ * up to the end of the warp reduction and from there to the opening of the next item.  This call
  * synchronises the device and copies the records of warps 0 .. warps-1 (at most 4096; warp = block * 8 + warp
- * in block) of the last launch to words_host[warps * 9].  `python -m paper_2605_14978_b200.timeline` prints a
+ * in block) of the last launch to words_host[warps * 11].  `python -m paper_2605_14978_b200.timeline` prints a
  * summary.  In the ordinary library: PPOW_ERR_UNSUPPORTED.
  */
 ppow_status ppow_timeline_read(uint64_t *words_host, size_t warps);

@@ -190,9 +190,9 @@ def ppow_checked_failures():
 
 
 def ppow_timeline_read(warps: int):
-    """(status, array [warps, 9] of uint64) from the timeline build; status PPOW_ERR_UNSUPPORTED otherwise."""
+    """(status, array [warps, 11] of uint64) from the timeline build; status PPOW_ERR_UNSUPPORTED otherwise."""
     import numpy as np
-    buf = np.zeros((int(warps), 9), dtype=np.uint64)
+    buf = np.zeros((int(warps), 11), dtype=np.uint64)
     st = load_library().ppow_timeline_read(ctypes.c_void_p(buf.ctypes.data), int(warps))
     return int(st), buf
 

@@ -13,13 +13,15 @@
 
 namespace ppow {
 
-// Timeline build (-DPPOW_TIMELINE): every warp of the bulk-copy kernel leaves eight 64-bit words behind --
+// Timeline build (-DPPOW_TIMELINE): every warp of the bulk-copy kernel leaves eleven 64-bit words behind --
 // start, first data and end (%globaltimer, ns), items and tiles done, SM id, cycles spent waiting for copies,
-// cycles spent in item ends -- plus its total cycles; ppow_timeline_read copies them out.  Costs a few
-// instructions per tile; the ordinary build has none of it.
+// cycles spent in item ends, its total cycles, and of the item-end cycles those up to the end of the warp
+// reduction and those from there to the opening of the next item; ppow_timeline_read copies them out.  Costs a
+// few instructions per tile; the ordinary build has none of it.
 #ifdef PPOW_TIMELINE
 constexpr int TIMELINE_WARPS = 4096;
-__device__ unsigned long long g_timeline[TIMELINE_WARPS * 9];
+constexpr int TIMELINE_WORDS = 11;
+__device__ unsigned long long g_timeline[TIMELINE_WARPS * TIMELINE_WORDS];
 __device__ __forceinline__ unsigned long long global_ns()
 {
     unsigned long long t;
@@ -389,7 +391,7 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     PPOW_TL(const unsigned long long tl_t0 = global_ns(); unsigned long long tl_t1 = 0; unsigned tl_items = 0, tl_tiles = 0;
-            long long tl_wait = 0, tl_end = 0; const long long tl_c0 = clock64();)
+            long long tl_wait = 0, tl_end = 0, tl_reduce = 0, tl_open = 0; const long long tl_c0 = clock64();)
     unsigned char *stages = pipe_smem + (size_t)warp * PIPE_STAGES * 2 * TILE_BYTES;
     const uint32_t stages_addr = smem_addr(stages);
     const uint32_t bars_addr = smem_addr(&full_bar[warp][0]);
@@ -514,6 +516,7 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
                 else
                     cand[j] = Fmt::none();
             RowPartial p = warp_reduce(acc);
+            PPOW_TL(const long long tl_e1 = clock64(); tl_reduce += tl_e1 - tl_e0;)
             // the consumer moves on to its next item while the re-read is in flight
             const uint32_t done = C.item;
             acc.reset();
@@ -521,6 +524,7 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
             const uint32_t nx = item_ring[warp][consumed % ITEM_RING];
             ++consumed;
             open_item<SHIFTED>(job, C, nx);
+            PPOW_TL(tl_open += clock64() - tl_e1;)
             int32_t arg = INT32_MAX;
             if (holder) {
 #pragma unroll
@@ -543,9 +547,10 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
     }
     PPOW_TL(const unsigned tl_w = blockIdx.x * PIPE_WARPS + warp;
             if (lane == 0 && tl_w < TIMELINE_WARPS) {
-                unsigned long long *o = g_timeline + (size_t)tl_w * 9;
+                unsigned long long *o = g_timeline + (size_t)tl_w * TIMELINE_WORDS;
                 o[0] = tl_t0; o[1] = tl_t1; o[2] = global_ns(); o[3] = tl_items; o[4] = tl_tiles; o[5] = sm_id();
                 o[6] = (unsigned long long)tl_wait; o[7] = (unsigned long long)tl_end; o[8] = (unsigned long long)(clock64() - tl_c0);
+                o[9] = (unsigned long long)tl_reduce; o[10] = (unsigned long long)tl_open;
             })
 }
 
@@ -1148,7 +1153,9 @@ extern "C" ppow_status ppow_timeline_read(uint64_t *words_host, size_t warps)
 #ifdef PPOW_TIMELINE
     if (warps > (size_t)TIMELINE_WARPS) return PPOW_ERR_INVALID_ARG;
     if (cudaDeviceSynchronize() != cudaSuccess) return PPOW_ERR_CUDA;
-    return cudaMemcpyFromSymbol(words_host, g_timeline, warps * 9 * sizeof(unsigned long long)) == cudaSuccess ? PPOW_OK : PPOW_ERR_CUDA;
+    return cudaMemcpyFromSymbol(words_host, g_timeline, warps * TIMELINE_WORDS * sizeof(unsigned long long)) == cudaSuccess
+               ? PPOW_OK
+               : PPOW_ERR_CUDA;
 #else
     (void)warps;
     return PPOW_ERR_UNSUPPORTED;   // not the timeline build

@@ -38,7 +38,7 @@ def run(w, label, dev):
         raise SystemExit("not the timeline build: run with PPOW_LIBRARY=timeline")
     t = t.astype(np.int64)
     t = t[t[:, 2] > 0]
-    t0, t1, t2, items, tiles, sm, wait, endc, total = (t[:, i] for i in range(9))
+    t0, t1, t2, items, tiles, sm, wait, endc, total, reduce, opened = (t[:, i] for i in range(11))
     base = t0.min()
     span = (t2.max() - base) / 1e3
     rows = int(x["valid_len"].sum()) if x["valid_len"] is not None else w.N * w.K
@@ -52,6 +52,9 @@ def run(w, label, dev):
     print("   items per warp               ", q(items), "  tiles per warp", q(tiles))
     print("   share of cycles waiting      ", q(wait / total), "  in item ends", q(endc / total))
     print("   cycles per item end          ", q(endc / np.maximum(items, 1)), "  cycles per tile", q((total - endc) / np.maximum(tiles, 1)))
+    it = np.maximum(items, 1)
+    print("   of an item end: up to the end of the warp reduction", q(reduce / it), "  reset + next item", q(opened / it),
+          "  argmax index + store", q((endc - reduce - opened) / it))
     grid = np.linspace(0, span, 41)
     done = [(np.clip((base + g * 1e3 - t1) / np.maximum(t2 - t1, 1), 0, 1) * tiles).sum() for g in grid]
     tile_bytes = 2 * 128 * 16
