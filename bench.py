@@ -528,7 +528,7 @@ def workload_entry(B, run, steps, sampler, peak, cores):
     and the parity counts of a small sample against the oracle."""
     w, mode = run.w, run.mode
     m = run.measure(steps, 3, trace=False)                       # the step as a caller runs it
-    m["kernel_ms"] = run.measure(min(steps, 100), 0)["kernel_ms"]    # and the row kernel alone
+    m["kernel_ms"] = run.measure(min(steps, 200), 0)["kernel_ms"]    # and the row kernel alone
     flags = B.ppow_read_error_flags(run.ws)
     entry = {"workload": w.name, "mode": mode, "N": w.N, "K": w.K, "V": w.V, "logits": w.dtype, "steps": steps,
              "ms_per_step": m["step_ms"], "windows_per_s": w.N / (m["step_ms"] * 1e-3),
