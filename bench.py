@@ -489,6 +489,23 @@ class Run:
         return {"elapsed_ms": elapsed_ms, "step_ms": elapsed_ms / steps, "kernel_ms": reduce_avg_ms, "t0": t0, "t1": t1,
                 "steps": steps}
 
+    def plain_kernel_ms(self, steps):
+        """Row kernel of the plain scoring pass (no training-side outputs) on this run's buffers, by events."""
+        B, x = self.B, self.x
+        out = B.alloc_outputs(self.w.N, self.w.K, self.dev)
+        call = B.ScoreCall(self.params, x["draft_logits"], x["target_logits"], x["draft_tokens"], x["uniforms"],
+                           x["valid_len"], None, out, self.ws)
+        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for a, b in pairs:
+            a.record(), b.record()
+        for _ in range(3):
+            call.launch(self.stream)
+        torch.cuda.synchronize()
+        for a, b in pairs:
+            call.launch(self.stream, a, b)
+        torch.cuda.synchronize()
+        return sum(a.elapsed_time(b) for a, b in pairs) / steps
+
     def free(self):
         for name in ("x", "out", "ws", "score_call", "select_call", "sel_ws", "selected"):
             setattr(self, name, None)
@@ -676,6 +693,8 @@ def run_ppow(args):
             mt = tr.measure(20, 3)
             fig = training_figures(tr, mt)
             fig["clocks"] = sampler.region(mt["t0"], mt["t1"])
+            plain_ms = tr.plain_kernel_ms(20)
+            fig["row_reduce_ms"], fig["row_reduce_gbs"] = plain_ms, tr.algo_bytes / (plain_ms * 1e-3) / 1e9
             training.append(fig)
             tr.free()
             del tr

@@ -47,8 +47,9 @@ def owner_of(window: int, n_total: int, world: int) -> Tuple[int, int]:
 def gather_scores(local_score: torch.Tensor, n_total: int, group=None) -> torch.Tensor:
     """All-gather the per-rank score shards into the global ``[n_total]`` score array (same on every rank).
 
-    The one exchange step of the path.  Equal shards use ``all_gather_into_tensor`` (NCCL: a single
-    collective on the current stream); ragged shards are padded to the largest shard and trimmed."""
+    The one exchange step of the path.  CUDA shards take one ``all_gather_into_tensor`` (NCCL, on the current
+    stream), ragged shards padded to the largest shard and trimmed afterwards; host tensors (gloo) use
+    ``all_gather``."""
     import torch.distributed as dist
     world = dist.get_world_size(group)
     rank = dist.get_rank(group)
@@ -57,23 +58,28 @@ def gather_scores(local_score: torch.Tensor, n_total: int, group=None) -> torch.
         raise ValueError("rank %d holds %d scores, its shard of %d windows has %d"
                          % (rank, local_score.numel(), n_total, sizes[rank]))
     local_score = local_score.contiguous()
-    if len(set(sizes)) == 1:
-        out = torch.empty((n_total,), dtype=local_score.dtype, device=local_score.device)
-        if local_score.is_cuda:
-            dist.all_gather_into_tensor(out, local_score, group=group)
-        else:
-            dist.all_gather(list(out.split(sizes[0])), local_score, group=group)
-        return out
     width = max(sizes)
-    padded = torch.zeros((width,), dtype=local_score.dtype, device=local_score.device)
-    padded[: sizes[rank]].copy_(local_score)
     if local_score.is_cuda:
+        # one code path for equal and ragged shards (so that a one-rank group exercises all of it): every rank
+        # contributes `width` scores, its own shard padded with zeros, in one NCCL all-gather on the current stream
+        if sizes[rank] == width:
+            padded = local_score
+        else:
+            padded = torch.zeros((width,), dtype=local_score.dtype, device=local_score.device)
+            padded[: sizes[rank]].copy_(local_score)
         flat = torch.empty((world * width,), dtype=local_score.dtype, device=local_score.device)
         dist.all_gather_into_tensor(flat, padded, group=group)
-        parts = list(flat.split(width))
-    else:
-        parts = [torch.empty_like(padded) for _ in range(world)]
-        dist.all_gather(parts, padded, group=group)
+        if len(set(sizes)) == 1:
+            return flat
+        return torch.cat([p[:s] for p, s in zip(flat.split(width), sizes)])
+    if len(set(sizes)) == 1:
+        out = torch.empty((n_total,), dtype=local_score.dtype, device=local_score.device)
+        dist.all_gather(list(out.split(sizes[0])), local_score, group=group)
+        return out
+    padded = torch.zeros((width,), dtype=local_score.dtype, device=local_score.device)
+    padded[: sizes[rank]].copy_(local_score)
+    parts = [torch.empty_like(padded) for _ in range(world)]
+    dist.all_gather(parts, padded, group=group)
     return torch.cat([p[:s] for p, s in zip(parts, sizes)])
 
 
