@@ -1,7 +1,8 @@
-// PPOW scoring pass: row-reduction kernels (the only HBM-heavy step: the bulk-copy pipeline kernel for
-// rows of whole 16-byte units, a scalar kernel for everything else), the per-window scan kernel, and the
-// host entry points ppow_score_windows(_traced) / ppow_score_workspace_bytes / ppow_read_error_flags /
-// ppow_selftest_wait_timeout.
+// PPOW scoring pass: row-reduction kernels (the only HBM-heavy step: the bulk-copy pipeline kernel, with
+// instances for rows of whole 16-byte units and for rows that start inside a unit, and a scalar kernel for
+// tensors at different offsets within a unit), the per-window scan kernel, the one-launch kernel for small
+// problems, and the host entry points ppow_score_windows(_traced) / ppow_score_workspace_bytes /
+// ppow_score_kernel_launches / ppow_read_error_flags / ppow_timeline_read / ppow_selftest_wait_timeout.
 #include "../../include/ppow.h"
 #include "ppow_device.cuh"
 #include "ppow_async.cuh"
@@ -170,9 +171,10 @@ __device__ __forceinline__ int32_t warp_min_i32(int32_t v)
     return r;
 }
 
-// ---- bulk-copy pipeline, one warp per work item (bf16, f16 or f32 rows of whole 16-byte units) -----
-// Each warp takes (row, segment) items from the work counter on its own; no block barrier is used after
-// set-up, so the warps of an SM drift apart.  The logits reach the warp through its own ring of
+// ---- bulk-copy pipeline, one warp per work item (bf16, f16 or f32; both tensors at the same offset within a
+// 16-byte unit) ----
+// Each warp takes work items on its own (its first by its index, the rest from the work counter); no block
+// barrier is used at all, so the warps of an SM drift apart.  The logits reach the warp through its own ring of
 // PIPE_STAGES shared-memory stages filled by bulk copies (cp.async.bulk + mbarrier): while the warp
 // computes on one tile, the copies of the next PIPE_STAGES - 1 tiles are in flight, across the end of
 // an item into the next one.  Loads never pause for the arithmetic, the end-of-item reduction or the
@@ -554,7 +556,7 @@ __global__ void __launch_bounds__(PIPE_WARPS * 32, PIPE_MIN_CTAS) row_reduce_pip
             })
 }
 
-// ---- generic path: any V, any alignment, f32 or bf16 -------------------------------------------
+// ---- scalar path: any V, any alignment, any storage type ----------------------------------------
 
 // One warp reduces logits [v0, v1) of a row with scalar coalesced loads: the loads of SCALAR_BATCH strides are
 // issued together (a lane would otherwise have one pair of loads in flight per trip), then folded one by one.
