@@ -443,12 +443,13 @@ def test_uniforms_just_outside_the_band_around_alpha(T, scale):
 
 def test_randomised_shapes_parameters_and_masks():
     """Property-style sweep: seeded random shapes (odd and even V, one position to 32, one window to dozens),
-    storage types, temperatures, costs, ragged masks and logit scales; everything is compared with the oracle."""
+    storage types, temperatures, costs, ragged masks, logit scales and base-pointer offsets; everything is compared
+    with the oracle."""
     rng = np.random.default_rng(2024)
-    for case in range(40):
+    for case in range(60):
         N = int(rng.integers(1, 40))
         K = int(rng.choice([1, 2, 3, 5, 8, 10, 12, 17, 32]))
-        V = int(rng.choice([2, 3, 8, 9, 64, 257, 1000, 1024, 4096 + 8, 5000, 20000, 40004]))
+        V = int(rng.choice([2, 3, 8, 9, 64, 257, 1000, 1024, 2049, 4096 + 8, 5000, 5001, 20000, 40004, 50257]))
         if N * K * V > 6_000_000:
             N = max(1, 6_000_000 // (K * V))
         dtype = [torch.bfloat16, torch.float32, torch.float16][int(rng.choice(3, p=[0.5, 0.25, 0.25]))]
@@ -456,6 +457,13 @@ def test_randomised_shapes_parameters_and_masks():
         c = float(rng.choice([0.0, 0.03, 0.12, 0.5]))
         scale = float(rng.choice([0.3, 2.0, 8.0]))
         x = _random_inputs(N, K, V, dtype, seed=1000 + case, sigma=float(rng.choice([0.0, 0.3, 1.5])), scale=scale)
+        off_t = int(rng.choice([0, 0, 1, 3]))                       # base pointers off a 16-byte boundary, mostly by the
+        off_d = off_t if rng.random() < 0.8 else int(rng.choice([0, 2]))   # same amount (else: the scalar row kernel)
+        if off_t or off_d:
+            for key, off in (("target_logits", off_t), ("draft_logits", off_d)):
+                flat = torch.full((N * K * V + 16,), 100.0, dtype=dtype, device=DEV)
+                flat[off:off + N * K * V].copy_(x[key].flatten())
+                x[key] = flat[off:off + N * K * V].view(N, K, V)
         if rng.random() < 0.5:
             x["valid_len"] = torch.from_numpy(rng.integers(0, K + 1, size=N).astype(np.int32)).to(DEV)
         if rng.random() < 0.3:                                       # drafted tokens that are the target's choice
