@@ -358,9 +358,10 @@ def test_status_codes_for_bad_arguments():
         B.select_windows(s, 11)
 
 
-def test_host_buffer_entry_point_matches_device_path_with_chunking():
+@pytest.mark.parametrize("V", [4096, 5001])                          # rows of whole units / rows that start inside a unit
+def test_host_buffer_entry_point_matches_device_path_with_chunking(V):
     w = W.scaled(W.WORKLOADS[3], 70)
-    w = dataclasses.replace(w, V=4096)
+    w = dataclasses.replace(w, V=V)
     x = W.generate(w, DEV)
     dev_out = run_gpu(x, "stochastic", w.c, w.temperature)
     dev_sel = B.select_windows(dev_out["score"], w.n_keep)
@@ -376,8 +377,15 @@ def test_host_buffer_entry_point_matches_device_path_with_chunking():
                                      scratch)
         torch.cuda.synchronize()
         for k, v in out_host.items():
-            assert torch.equal(v, dev_out[k].cpu()), (chunk, k)
-        assert torch.equal(sel_host, dev_sel.cpu())
+            if V % 8 == 0 or not v.dtype.is_floating_point:      # whole units: the same lanes add the same logits
+                assert torch.equal(v, dev_out[k].cpu()), (chunk, k)
+            else:                                                # rows start at other offsets in a staged chunk than in
+                torch.testing.assert_close(v, dev_out[k].cpu(), rtol=1e-5, atol=1e-6, msg=str((chunk, k)))   # the batch
+        if V % 8 == 0:
+            assert torch.equal(sel_host, dev_sel.cpu())
+        else:
+            want = oracle.select_windows(out_host["score"].numpy().astype(np.float64), w.n_keep)
+            np.testing.assert_array_equal(sel_host.numpy(), want)
         assert int(mask_host.sum()) == w.n_keep
     with pytest.raises(B.PpowError):
         B.ppow_score_and_select_host(params, host["draft_logits"], host["target_logits"], host["draft_tokens"],
