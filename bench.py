@@ -667,6 +667,18 @@ def run_ppow(args):
         e2e = {"value": run.n_total * e2e_steps / e2e_s, "unit": "windows/s", "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": 1e3 * e2e_s / e2e_steps,
                "note": "ppow_score_and_select_host: pinned host logits copied to the device inside the timed region"}
+        # the same call with scratch for an eighth of the windows at a time (eight staged chunks on the one stream)
+        if solo and N >= 64:
+            small = B.alloc_workspace(B.ppow_host_scratch_bytes(run.params, N // 8), dev)
+            scratch = small
+            e2e_step()
+            t0 = time.perf_counter()
+            for _ in range(3):
+                e2e_step()
+            dt = (time.perf_counter() - t0) / 3
+            e2e["chunked"] = {"chunk_windows": N // 8, "scratch_bytes": int(small.numel()), "value": run.n_total / dt,
+                              "ms_per_step": 1e3 * dt}
+            del small
         del host, out_host, scratch
 
     # ---- one entry per other workload (generated, timed, checked and freed one at a time)
