@@ -638,6 +638,7 @@ struct ScanJob {
     int32_t N, K, V, dtype, mode;
     float s;         // log2(e)/T as used by the row reduction
     float c, eta, eps;
+    double ln_v;     // ln V
 };
 
 __device__ __forceinline__ double raw_logit(const void *base, int32_t dtype, size_t idx)
@@ -715,13 +716,37 @@ __device__ __forceinline__ RowSums shfl_sums(const RowSums &m, int src_lane, boo
     return r;
 }
 
-// One warp scores window n, lane = position.  `m`: the merged reductions of this lane's row (unused by
-// lanes beyond the window's valid length).
-__device__ __forceinline__ void scan_window(const ScanJob &job, const int32_t n, const int lane, const RowSums &m)
+// What the scan needs about the drafted token of one position: read ahead of the merge of the row's parts, so
+// that these dependent loads (token id, then the two logits at that id) are in flight meanwhile.
+struct TokenRead {
+    int32_t tok;
+    bool in_range;
+    double a_tok, b_tok, u;
+};
+
+__device__ __forceinline__ TokenRead read_token(const ScanJob &job, const int32_t n, const int lane, const int32_t L)
+{
+    TokenRead r = {0, false, 0.0, 0.0, 0.0};
+    if (lane >= L) return r;
+    const size_t row = (size_t)n * job.K + lane;
+    r.tok = __ldg(job.tokens + row);
+    r.in_range = r.tok >= 0 && r.tok < job.V &&
+                 PPOW_CHECK(row < (size_t)job.N * job.K && row * job.V + r.tok < (size_t)job.N * job.K * job.V, 202,
+                            &job.header->error_flags);
+    if (r.in_range) {
+        r.a_tok = raw_logit(job.target, job.dtype, row * job.V + r.tok);
+        r.b_tok = raw_logit(job.draft, job.dtype, row * job.V + r.tok);
+    }
+    if (job.mode != PPOW_GREEDY) r.u = (double)__ldg(job.uniforms + row);
+    return r;
+}
+
+// One warp scores window n, lane = position.  `m`: the merged reductions of this lane's row, `tr`: its drafted
+// token (both unused by lanes beyond the window's valid length L).
+__device__ __forceinline__ void scan_window(const ScanJob &job, const int32_t n, const int lane, const int32_t L,
+                                            const RowSums &m, const TokenRead &tr)
 {
     const int32_t K = job.K;
-    int32_t L = job.valid_len ? __ldg(job.valid_len + n) : K;
-    L = max(0, min(L, K));
     const bool active = lane < L;
     const double LN2 = 0.69314718055994530942;
 
@@ -731,7 +756,6 @@ __device__ __forceinline__ void scan_window(const ScanJob &job, const int32_t n,
     int flag = 0;
 
     if (active) {
-        const size_t row = (size_t)n * K + lane;
         const double Ra = m.Ra, Rb = m.Rb, Sa = m.Sa, Sb = m.Sb, E = m.E, D = m.D, Bv = m.B;
         const float mx = m.mx;
         const int32_t arg = m.arg;
@@ -742,24 +766,21 @@ __device__ __forceinline__ void scan_window(const ScanJob &job, const int32_t n,
         kl_rev = (-Bv / Sb - l2Sb + l2Sa) * LN2;              // KL(Q || P), nats (meaningful only if B was accumulated)
         o_lse_p = (float)((Ra + l2Sa) * LN2);
         o_lse_q = (float)((Rb + l2Sb) * LN2);
-        double C = 1.0 - H / log((double)job.V);
+        double C = 1.0 - H / job.ln_v;
         C = fmin(1.0, fmax(0.0, C));
         crit = C * KL;
         const double lmax2 = fma((double)mx, s, -Ra) - l2Sa;   // log2 P(argmax); explicit fma: same rounding as lp2
 
-        const int32_t tok = __ldg(job.tokens + row);
+        const int32_t tok = tr.tok;
         double lq, lp2 = -INFINITY;
-        if (tok < 0 || tok >= job.V ||
-            !PPOW_CHECK(row < (size_t)job.N * job.K && row * job.V + tok < (size_t)job.N * job.K * job.V, 202,
-                        &job.header->error_flags)) {
+        if (!tr.in_range) {
             atomicOr(&job.header->error_flags, (unsigned)PPOW_FLAG_TOKEN_RANGE);
             lp = -INFINITY;
             lq = -INFINITY;
             flag = 0;
             o_nabla = INFINITY;
         } else {
-            const double a_tok = raw_logit(job.target, job.dtype, row * job.V + tok);
-            const double b_tok = raw_logit(job.draft, job.dtype, row * job.V + tok);
+            const double a_tok = tr.a_tok, b_tok = tr.b_tok;
             lp2 = fma(a_tok, s, -Ra) - l2Sa;
             lp = lp2 * LN2;
             lq = (fma(b_tok, s, -Rb) - l2Sb) * LN2;
@@ -768,7 +789,7 @@ __device__ __forceinline__ void scan_window(const ScanJob &job, const int32_t n,
                 flag = (tok == arg);
             } else {
                 const double alpha = fmin(1.0, exp(lp - lq));
-                flag = ((double)__ldg(job.uniforms + row) <= alpha);
+                flag = (tr.u <= alpha);
             }
         }
         gap = (lmax2 - lp2) * LN2;   // differenced before scaling: exactly 0 when the token is the argmax
@@ -838,6 +859,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
     int kp = 1;
     while (kp < job.K) kp <<= 1;
     const int G = 32 / kp, r = lane / G, sub = lane & (G - 1);
+    const TokenRead tr = read_token(job, n, lane, L);   // in flight while the parts are merged
     if (r < L) row_items(job.plan, (uint32_t)n * (uint32_t)job.K + (uint32_t)r, first_part, parts);
     if (!PPOW_CHECK((size_t)first_part + parts <= job.plan.item_begin[PLAN_CLASSES] && parts <= (1 << MAX_SHIFT), 204,
                     &job.header->error_flags))
@@ -845,7 +867,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
     RowSums m = merge_partials(job.partials + first_part, parts, sub, G);
     for (int o = G >> 1; o > 0; o >>= 1) fold_sums(m, shfl_sums(m, o, true));
     m = shfl_sums(m, (lane * G) & 31, false);
-    scan_window(job, n, lane, m);
+    scan_window(job, n, lane, L, m, tr);
 }
 
 // ---- small problems: the whole pass in one launch ---------------------------------------------------
@@ -877,7 +899,10 @@ __global__ void __launch_bounds__(1024) score_small_kernel(const RowJob rj, cons
         }
     }
     __syncthreads();
-    if (warp == 0) scan_window(sj, n, lane, merge_partials(&parts[lane < rj.K ? lane : 0], lane < L ? 1 : 0));
+    if (warp == 0) {
+        const TokenRead tr = read_token(sj, n, lane, L);
+        scan_window(sj, n, lane, L, merge_partials(&parts[lane < rj.K ? lane : 0], lane < L ? 1 : 0), tr);
+    }
 }
 
 // ---- self-test of the bounded wait ----------------------------------------------------------------
@@ -1046,6 +1071,7 @@ extern "C" ppow_status ppow_score_windows_traced(const ppow_params *params,
     sj.out = *out;
     sj.N = params->N; sj.K = params->K; sj.V = params->V; sj.dtype = params->dtype; sj.mode = params->mode;
     sj.plan = plan; sj.s = s; sj.c = params->c; sj.eta = params->eta; sj.eps = params->eps;
+    sj.ln_v = log((double)params->V);
     const bool rev = out->kl_rev != nullptr || out->kl_rev_mean != nullptr;
 
     // a few megabytes of short rows: one launch for the whole pass (the events bracket that launch)
