@@ -717,17 +717,20 @@ __device__ __forceinline__ RowSums shfl_sums(const RowSums &m, int src_lane, boo
 }
 
 // What the scan needs about the drafted token of one position: read ahead of the merge of the row's parts, so
-// that these dependent loads (token id, then the two logits at that id) are in flight meanwhile.
+// that these dependent loads (token id, then the two logits at that id) are in flight meanwhile.  Read for every
+// position of the window, valid or not (the arrays hold K entries per window; a masked position's token is only
+// looked at if it happens to be a vocabulary index, and is never scored), so that nothing here waits for the
+// window's valid length.
 struct TokenRead {
     int32_t tok;
     bool in_range;
     double a_tok, b_tok, u;
 };
 
-__device__ __forceinline__ TokenRead read_token(const ScanJob &job, const int32_t n, const int lane, const int32_t L)
+__device__ __forceinline__ TokenRead read_token(const ScanJob &job, const int32_t n, const int lane)
 {
     TokenRead r = {0, false, 0.0, 0.0, 0.0};
-    if (lane >= L) return r;
+    if (lane >= job.K) return r;
     const size_t row = (size_t)n * job.K + lane;
     r.tok = __ldg(job.tokens + row);
     r.in_range = r.tok >= 0 && r.tok < job.V &&
@@ -851,22 +854,24 @@ __global__ void __launch_bounds__(SCAN_THREADS) window_scan_kernel(const ScanJob
     if (n >= job.N) return;
     uint32_t first_part = 0;
     int parts = 0;
-    int32_t L = job.valid_len ? __ldg(job.valid_len + n) : job.K;
-    L = max(0, min(L, job.K));
     // G lanes share the merge of one row's parts (rows near the end of the launch are cut into up to 32 items):
     // lanes [r*G, r*G + G) take parts sub, sub + G, ... of row r, fold their results together, and lane t, which
     // scores position t, fetches row t's sums from lane t*G
     int kp = 1;
     while (kp < job.K) kp <<= 1;
     const int G = 32 / kp, r = lane / G, sub = lane & (G - 1);
-    const TokenRead tr = read_token(job, n, lane, L);   // in flight while the parts are merged
-    if (r < L) row_items(job.plan, (uint32_t)n * (uint32_t)job.K + (uint32_t)r, first_part, parts);
+    int32_t L = job.valid_len ? __ldg(job.valid_len + n) : job.K;   // first needed after the merge
+    const TokenRead tr = read_token(job, n, lane);                    // in flight while the parts are merged
+    // every row of the window is merged, valid or not (a masked row's slots hold whatever an earlier call left
+    // there; the result is dropped below), so that the loads do not wait for the valid length
+    if (r < job.K) row_items(job.plan, (uint32_t)n * (uint32_t)job.K + (uint32_t)r, first_part, parts);
     if (!PPOW_CHECK((size_t)first_part + parts <= job.plan.item_begin[PLAN_CLASSES] && parts <= (1 << MAX_SHIFT), 204,
                     &job.header->error_flags))
         parts = 0;
     RowSums m = merge_partials(job.partials + first_part, parts, sub, G);
     for (int o = G >> 1; o > 0; o >>= 1) fold_sums(m, shfl_sums(m, o, true));
     m = shfl_sums(m, (lane * G) & 31, false);
+    L = max(0, min(L, job.K));
     scan_window(job, n, lane, L, m, tr);
 }
 
@@ -900,7 +905,7 @@ __global__ void __launch_bounds__(1024) score_small_kernel(const RowJob rj, cons
     }
     __syncthreads();
     if (warp == 0) {
-        const TokenRead tr = read_token(sj, n, lane, L);
+        const TokenRead tr = read_token(sj, n, lane);
         scan_window(sj, n, lane, L, merge_partials(&parts[lane < rj.K ? lane : 0], lane < L ? 1 : 0), tr);
     }
 }
