@@ -553,8 +553,12 @@ def workload_entry(B, run, steps, sampler, peak, cores, with_oracle=True):
              "kernel_ms": m["kernel_ms"], "valid_row_bytes": run.algo_bytes,
              "logit_gbs": run.algo_bytes / (m["kernel_ms"] * 1e-3) / 1e9,
              "frac": run.algo_bytes / (m["kernel_ms"] * 1e-3) / 1e9 / peak,
+             "frac_of_nominal_8TBs": run.algo_bytes / (m["kernel_ms"] * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
              "hbm_figure": run.algo_bytes > 4e8, "clocks": sampler.region(m["t0"], m["t1"]), "error_flags": flags}
-    entry["parity"] = oracle_leg(B, run, PARITY_SAMPLE_WINDOWS, cores)[2] if with_oracle else None
+    entry["parity"] = entry["oracle"] = None
+    if with_oracle:
+        dt, nw, entry["parity"] = oracle_leg(B, run, PARITY_SAMPLE_WINDOWS, cores)
+        entry["oracle"] = {"windows_per_s": nw / dt, "cores": cores, "sample": "first %d windows" % nw}
     return entry
 
 
