@@ -223,7 +223,7 @@ def dist_setup(n_gpus):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world > 1 or "RANK" in os.environ:    # launched by torch.distributed.run, even with one rank: use the collective
+    if world > 1 or "TORCHELASTIC_RUN_ID" in os.environ:    # launched by torch.distributed.run, even with one rank: use the collective
         import torch.distributed as dist
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         os.environ.setdefault("MASTER_PORT", "29500")
