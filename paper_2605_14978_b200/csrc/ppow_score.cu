@@ -45,7 +45,8 @@ constexpr int UNROLL = 4;          // 16-byte units per lane per tensor in one t
 constexpr int TILE_UNITS = 32 * UNROLL;       // 16-byte units per tile per tensor
 constexpr int MAX_SHIFT = 5;       // a row is split into at most 2^5 work items
 constexpr int PLAN_CLASSES = 5;    // row classes of the work plan: items of at most 64, 32, 16, 8, 4 tiles
-constexpr int PLAN_K = 1;          // an item is at most 1/PLAN_K of a resident warp's share of the work still to hand out
+// an item is at most 1/1 (rows shorter than 64 tiles) or 2/3 (longer rows) of a resident warp's share of the work
+// still to hand out
 constexpr size_t WS_HEADER_BYTES = 256;
 constexpr size_t SMALL_ROW_BYTES = 4096;        // rows up to this long (at most two tiles) in
 constexpr size_t SMALL_TOTAL_BYTES = 4u << 20;  // calls up to this many logit bytes take the one-launch kernel
@@ -948,8 +949,12 @@ static bool params_ok(const ppow_params *p)
 // the warps run at speeds that differ by +-20 % and finish their last items spread over one item's
 // duration, which on a launch of a few hundred microseconds is 10-15 % of the time.  So the items shrink
 // as the work runs out (guided self-scheduling, fixed ahead of time): a row whose distance from the last
-// row leaves R tiles of work still to hand out is cut into items of at most R / (PLAN_K * resident warps)
-// tiles, rounded down to 64, 32, 16, 8 or 4.
+// row leaves R tiles of work still to hand out is cut into items of at most R / (resident warps) tiles (a warp's
+// share of what is left), rounded down to 64, 32, 16, 8 or 4.  Warps run at speeds that differ by +-20 % (by SM), so a slow warp
+// that takes an item of a warp's whole remaining share ends late by a fifth of that item; on rows of 64 tiles
+// and more, where an item end is cheap next to the item, the items therefore shrink half an item length earlier
+// (measured: +2 % on a 256-window launch of the headline shape, within noise on the full workloads; on the short rows of the
+// Vicuna-like workload the extra item ends cost 1 %, so those keep the whole share).
 constexpr int64_t WORKER_WARPS = 148 * PIPE_MIN_CTAS * PIPE_WARPS;   // resident warps of the bulk-copy kernel on a B200
 
 static int shift_for(int64_t tiles, int64_t item_tiles)
@@ -966,14 +971,15 @@ static WorkPlan make_plan(const ppow_params *p)
     const int64_t tile_logits = (int64_t)TILE_UNITS * (p->dtype == PPOW_F32 ? 4 : 8);
     const int64_t tiles = ((int64_t)p->V + tile_logits - 1) / tile_logits;   // per row
     plan.tiles = (int32_t)tiles;
-    // class i holds items of at most 64 >> i tiles; it starts at the first row from which at least
-    // PLAN_K * (64 >> i) * WORKER_WARPS tiles are still to come, and ends where the next class starts
+    // class i holds items of at most 64 >> i tiles; it ends (and the next class starts) at the first row from
+    // which fewer than margin * (64 >> i) * WORKER_WARPS tiles are still to come
     uint32_t item = 0;
     int64_t row = 0;
     for (int i = 0; i < PLAN_CLASSES; ++i) {
         int64_t end = rows;   // first row of the next class
         if (i + 1 < PLAN_CLASSES) {
-            const int64_t from_end = (PLAN_K * (int64_t)(64 >> i) * WORKER_WARPS + tiles - 1) / tiles;
+            const int64_t margin_num = tiles >= 64 ? 3 : 2;   // halves: 3/2 of the item length for long rows, else 1
+            const int64_t from_end = (margin_num * (int64_t)(64 >> i) * WORKER_WARPS / 2 + tiles - 1) / tiles;
             end = rows > from_end ? rows - from_end : 0;
         }
         if (end < row) end = row;
